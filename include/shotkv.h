@@ -1,0 +1,216 @@
+/*
+ * shotkv.h -- C ABI of the ShotKV hot path for NVIDIA B200 (sm_100a).
+ *
+ * ShotKV (arXiv 2502.01941, Section 5.1 and Algorithm 1) compresses the KV cache
+ * of a few-shot prompt once after prefill, keeping whole shots ("semantic units")
+ * ranked by the attention they receive, and compresses the decode-side cache
+ * token by token while generating.  This library is that path and nothing else.
+ *
+ * Conventions for every call
+ *   - "device" pointers are CUDA global memory of the context's device, "host"
+ *     pointers are ordinary process memory.  The caller owns every buffer,
+ *     workspaces included; the library owns only the shotkv_ctx.
+ *   - bf16 tensors are raw 16-bit patterns (shotkv_bf16).  Rows of d contiguous
+ *     elements; all tensors dense in the index order written beside them; base
+ *     addresses 16-byte aligned.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = the
+ *     legacy default stream); calls return without synchronising unless stated.
+ *   - Return value: 0 = ok, negative = error (nothing useful was enqueued),
+ *     positive = warning (the work was enqueued).  shotkv_last_error() gives text.
+ *   - There is no CPU fallback: without a CUDA device every compute call fails.
+ *
+ * Index names: B prompts, L layers, H query heads, Hkv KV heads (G = H/Hkv),
+ * d head dimension (64 or 128), N prompt tokens, W observation-window rows
+ * (the last W prompt positions), S shots.  Shot i covers tokens
+ * [off[i], off[i+1]) and has k_i = off[i+1]-off[i] >= 1 tokens; tokens before
+ * off[0] and from off[S] on (the question, which contains the window) are
+ * always kept and count against the budget.
+ */
+#ifndef SHOTKV_H_
+#define SHOTKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define SHOTKV_API __attribute__((visibility("default")))
+#else
+#define SHOTKV_API
+#endif
+
+typedef struct shotkv_ctx shotkv_ctx;
+typedef uint16_t shotkv_bf16;
+
+typedef struct {
+    int32_t B, L, H, Hkv, d, N, W, S;
+} shotkv_dims;
+
+typedef struct {
+    float   r_p;              /* prefill ratio: N_budget = floor(r_p * N) tokens per layer        */
+    int32_t select_mode;      /* 0: stop at the first shot that overflows; 1: skip it and go on   */
+    float   r_d;              /* decode ratio: k = floor(r_d * T) after T generated tokens        */
+    int32_t recompress_every; /* decode: evict every this many steps (1 = every step)             */
+    int32_t protect_recent;   /* must be 0 (the paper's rule protects nothing)                    */
+} shotkv_policy;
+
+enum {
+    SHOTKV_OK = 0,
+    SHOTKV_ERR_INVALID_ARG = -1,
+    SHOTKV_ERR_UNSUPPORTED_SHAPE = -2,
+    SHOTKV_ERR_BAD_OFFSETS = -3,          /* not increasing, empty shot, off[0] < 0 or off[S] > N-W  */
+    SHOTKV_ERR_WORKSPACE_TOO_SMALL = -4,
+    SHOTKV_ERR_CUDA = -5,
+    SHOTKV_ERR_TIMEOUT = -6,              /* a bounded device-side wait gave up                     */
+    SHOTKV_WARN_BUDGET_BELOW_ALWAYS_KEPT = 1 /* some prompt's always-kept tokens exceed floor(r_p*N);
+                                                only they are kept for that prompt                  */
+};
+
+/* Bit set in `flags` of shotkv_prefill_compress. */
+#define SHOTKV_FLAG_TOKEN_IMPORTANCE 1u   /* also produce per-token importance (two passes over K) */
+
+/* ---- context ------------------------------------------------------------------------------- */
+
+/* Creates a context bound to CUDA device `device`.  Fails with SHOTKV_ERR_CUDA when there is no
+ * such device or it is not compute capability 10.x.  */
+SHOTKV_API int shotkv_create(shotkv_ctx** ctx, int device);
+SHOTKV_API void shotkv_destroy(shotkv_ctx* ctx);
+/* Text of the last error or warning recorded on this context (never NULL; "" if none). */
+SHOTKV_API const char* shotkv_last_error(const shotkv_ctx* ctx);
+/* Library version string. */
+SHOTKV_API const char* shotkv_version(void);
+
+/* ---- host helpers (no GPU needed) ---------------------------------------------------------- */
+
+/* N_budget = floor(r_p * N), the product taken in double with r_p as the float it is
+ * (Section 5.1: budget r_p x |KV_prefill|, |KV_prefill| = all N prompt tokens).  */
+SHOTKV_API int32_t shotkv_budget_tokens(const shotkv_dims* dims, const shotkv_policy* policy);
+/* Rows to allocate per (b,l[,hkv]) for kept_idx / Kc / Vc: max(N_budget, largest always-kept
+ * count over the B prompts).  offsets_host [B][S+1].  Negative error code on bad input.  */
+SHOTKV_API int32_t shotkv_kept_capacity(const shotkv_dims* dims, const shotkv_policy* policy,
+                             const int32_t* offsets_host);
+/* Checks shapes and offsets exactly as the compute calls do.  Returns 0, a negative error, or
+ * SHOTKV_WARN_BUDGET_BELOW_ALWAYS_KEPT.  policy and offsets_host may be NULL to check dims only. */
+SHOTKV_API int shotkv_validate(const shotkv_dims* dims, const shotkv_policy* policy,
+                    const int32_t* offsets_host);
+/* Bytes of device workspace that the prefill calls below need for `dims` (any of them; one
+ * buffer of this size serves all).  0 on invalid dims.  */
+SHOTKV_API size_t shotkv_workspace_bytes(const shotkv_dims* dims);
+
+/* ---- prefill (Algorithm 1, Phase 1) -------------------------------------------------------- */
+
+/* Window attention and column-sum: the alpha of the prefill score equation (Section 5.1).
+ * For every (b, l, kv head g) the R = G*W window rows (heads g*G..g*G+G-1, positions N-W..N-1)
+ * attend causally to the prompt keys with scale 1/sqrt(d); every row is a softmax over the keys at
+ * or before its own position; token_importance[b][l][g][t] is the sum of column t over those rows.
+ *   Qwin  device [B][L][H][W][d] bf16      K  device [B][L][Hkv][N][d] bf16
+ *   token_importance  device [B][L][Hkv][N] f32 (written in full)
+ *   ws    device workspace of >= shotkv_workspace_bytes(dims) bytes, 256-byte aligned
+ * Supported: d in {64,128}, G*W <= 256, W <= N.  */
+SHOTKV_API int shotkv_prefill_score(shotkv_ctx* ctx, const shotkv_dims* dims,
+                         const shotkv_bf16* Qwin, const shotkv_bf16* K,
+                         float* token_importance, void* ws, size_t ws_bytes, void* stream);
+
+/* Per-shot score and whole-shot selection (prefill score equation, TopK equation and its budget
+ * constraint in Section 5.1; "sort ... select shots until" in Algorithm 1).
+ *   Score(s_i) = (1/k_i) * sum_{t in s_i} sum_{g} token_importance[b][l][g][t]      per (b, l)
+ * Shots are ordered by (score descending, index ascending) and kept per `select_mode` while the
+ * kept shot tokens fit floor(r_p*N) minus the always-kept tokens.  Scores must be finite.
+ *   token_importance device [B][L][Hkv][N] f32, or NULL to rank the shot_scores already in place
+ *   offsets_host     host   [B][S+1] int32 (validated; uploaded into ws on `stream`)
+ *   shot_scores      device [B][L][S] f32   (output; input when token_importance is NULL)
+ *   keep             device [B][L][S] u8    1 = shot kept
+ *   kept_idx         device [B][L][Mcap] i32 kept token positions ascending, -1 beyond kept_count
+ *   kept_count       device [B][L] i32
+ *   Mcap >= shotkv_kept_capacity(...).  */
+SHOTKV_API int shotkv_select_shots(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_policy* policy,
+                        const float* token_importance, const int32_t* offsets_host,
+                        float* shot_scores, uint8_t* keep, int32_t* kept_idx, int32_t* kept_count,
+                        int32_t Mcap, void* ws, size_t ws_bytes, void* stream);
+
+/* Compress (Section 5.1, Compress equation): gathers the kept rows of every KV head of a layer.
+ *   Kc[b][l][g][j] = K[b][l][g][kept_idx[b][l][j]]  for j < kept_count[b][l]; same for V.
+ *   K, V   device [B][L][Hkv][N][d] bf16     Kc, Vc  device [B][L][Hkv][Mcap][d] bf16
+ * Rows j >= kept_count[b][l] of Kc/Vc are left untouched.  Bit-exact copy.  */
+SHOTKV_API int shotkv_compact_kv(shotkv_ctx* ctx, const shotkv_dims* dims,
+                      const shotkv_bf16* K, const shotkv_bf16* V,
+                      const int32_t* kept_idx, const int32_t* kept_count, int32_t Mcap,
+                      shotkv_bf16* Kc, shotkv_bf16* Vc, void* stream);
+
+/* The whole of Phase 1 in one call: score, select, compact.  Without
+ * SHOTKV_FLAG_TOKEN_IMPORTANCE the shot scores are formed directly from per-shot partial sums
+ * (K is streamed once and per-token importance is never materialised; token_importance is
+ * ignored and may be NULL); with it the call equals the three calls above in sequence.
+ * Arguments as in those calls.  */
+SHOTKV_API int shotkv_prefill_compress(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_policy* policy,
+                            const shotkv_bf16* Qwin, const shotkv_bf16* K, const shotkv_bf16* V,
+                            const int32_t* offsets_host,
+                            float* shot_scores, uint8_t* keep, int32_t* kept_idx,
+                            int32_t* kept_count, int32_t Mcap,
+                            shotkv_bf16* Kc, shotkv_bf16* Vc,
+                            float* token_importance, uint32_t flags,
+                            void* ws, size_t ws_bytes, void* stream);
+
+/* Same, for callers whose tensors live in HOST memory (pinned memory makes the copies
+ * asynchronous).  Copies Qwin/K/V to the device arena, runs Phase 1, copies the results back, all
+ * on `stream`; returns after enqueueing.  Outputs with a NULL host pointer are not copied back.
+ *   arena  device buffer of >= shotkv_host_arena_bytes(dims, Mcap) bytes, 256-byte aligned
+ * The host outputs are valid once `stream` has been synchronised.  */
+SHOTKV_API size_t shotkv_host_arena_bytes(const shotkv_dims* dims, int32_t Mcap);
+SHOTKV_API int shotkv_prefill_compress_host(shotkv_ctx* ctx, const shotkv_dims* dims,
+                                 const shotkv_policy* policy,
+                                 const shotkv_bf16* Qwin_host, const shotkv_bf16* K_host,
+                                 const shotkv_bf16* V_host, const int32_t* offsets_host,
+                                 float* shot_scores_host, uint8_t* keep_host,
+                                 int32_t* kept_idx_host, int32_t* kept_count_host, int32_t Mcap,
+                                 shotkv_bf16* Kc_host, shotkv_bf16* Vc_host,
+                                 void* arena, size_t arena_bytes, void* stream);
+
+/* ---- decode (Algorithm 1, Phase 2) --------------------------------------------------------- */
+
+/* Decode-side cache of B sequences x L layers.  The caller allocates the device arrays and fills
+ * the struct through shotkv_decode_init; the library updates T and n_dec on the host.  Every
+ * sequence generates one token per step, so T and n_dec are the same for all (b, l).  */
+typedef struct {
+    shotkv_dims   dims;        /* B, L, H, Hkv, d are used                                         */
+    shotkv_policy policy;      /* r_d, recompress_every are used                                   */
+    int32_t Dcap;              /* rows per (b,l,g) of Kd/Vd; needs >= n_dec+1 at every step         */
+    int32_t Mcap;              /* rows per (b,l,g) of the compressed prefill keys Kc                */
+    int32_t T;                 /* tokens generated so far                                          */
+    int32_t n_dec;             /* decode entries currently held per (b,l)                          */
+    shotkv_bf16* Kd;           /* device [B][L][Hkv][Dcap][d]                                      */
+    shotkv_bf16* Vd;           /* device [B][L][Hkv][Dcap][d]                                      */
+    float*   acc;              /* device [B][L][Dcap]  accumulated Score_decoding per entry        */
+    int32_t* born;             /* device [B][L][Dcap]  generation step (0-based) of each entry     */
+    void*    ws;               /* device workspace, >= shotkv_decode_workspace_bytes()             */
+    size_t   ws_bytes;
+} shotkv_decode_state;
+
+SHOTKV_API size_t shotkv_decode_workspace_bytes(const shotkv_dims* dims, int32_t Dcap);
+/* Smallest Dcap that never overflows over `steps` steps under `policy`. */
+SHOTKV_API int32_t shotkv_decode_capacity(const shotkv_policy* policy, int32_t steps);
+/* Validates and fills `state` (T = n_dec = 0).  Touches no device memory.  */
+SHOTKV_API int shotkv_decode_init(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_policy* policy,
+                       int32_t Dcap, int32_t Mcap, shotkv_bf16* Kd, shotkv_bf16* Vd, float* acc,
+                       int32_t* born, void* ws, size_t ws_bytes, shotkv_decode_state* state);
+
+/* One generation step for all (b, l) (decoding score equation and TopK rule of Section 5.1):
+ *   1. append k_new/v_new as decode entry n_dec with score 0; T += 1;
+ *   2. for every query head, softmax of q.k/sqrt(d) over the kept prefill keys Kc[..][0..M) and
+ *      all decode keys together (M = kept_count[b][l]); acc[j] += sum over the H heads of the
+ *      weight on decode entry j;
+ *   3. if T % recompress_every == 0: keep the k = min(n_dec, floor(r_d*T)) entries greatest in
+ *      (acc descending, index ascending), compacted in index order (Kd, Vd, acc, born).
+ *   q device [B][L][H][d] bf16;  k_new, v_new device [B][L][Hkv][d] bf16;
+ *   Kc device [B][L][Hkv][Mcap][d] bf16;  kept_count device [B][L] i32.  */
+SHOTKV_API int shotkv_decode_step(shotkv_ctx* ctx, shotkv_decode_state* state,
+                       const shotkv_bf16* q, const shotkv_bf16* k_new, const shotkv_bf16* v_new,
+                       const shotkv_bf16* Kc, const int32_t* kept_count, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SHOTKV_H_ */

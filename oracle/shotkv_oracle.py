@@ -171,15 +171,10 @@ class DecodeOracle:
         self.born: list[int] = []
         self.T = 0
 
-    def step(self, q: np.ndarray, k_new: np.ndarray, v_new: np.ndarray, decide_acc=None):
-        """q [H, d], k_new/v_new [Hkv, d].  Appends the new token, adds this step's attention
-        weights (softmax over the prefill-kept and decode keys together) to the decode entries'
-        scores, and every R steps keeps the top floor(r_d*T) decode entries.
-
-        `decide_acc`, if given, replaces the scores *for the eviction decision only* (used by
-        lock-step parity tests to take the decision in the kernel's precision).
-        Returns the list of evicted entry indices (positions in the pre-eviction region).
-        """
+    def accumulate(self, q: np.ndarray, k_new: np.ndarray, v_new: np.ndarray) -> None:
+        """q [H, d], k_new/v_new [Hkv, d].  Appends the new token as a decode entry with score 0,
+        then adds this step's attention weights -- each head's softmax over the prefill-kept and
+        decode keys together, the new token included -- to the decode entries' scores."""
         q = np.asarray(q, dtype=np.float64)
         self.Kd.append(np.asarray(k_new, dtype=np.float64))
         self.Vd.append(np.asarray(v_new))
@@ -197,18 +192,37 @@ class DecodeOracle:
             add += a[self.M:]
         for j in range(n):
             self.acc[j] += add[j]
-        evicted: list[int] = []
-        if self.T % self.R == 0:
-            k = min(n, int(math.floor(self.r_d * self.T)))
-            sc = self.acc if decide_acc is None else list(decide_acc)
-            order = sorted(range(n), key=lambda j: (-sc[j], j))
-            kept = sorted(order[:k])
-            evicted = sorted(order[k:])
-            self.Kd = [self.Kd[j] for j in kept]
-            self.Vd = [self.Vd[j] for j in kept]
-            self.acc = [self.acc[j] for j in kept]
-            self.born = [self.born[j] for j in kept]
+
+    def eviction_due(self) -> bool:
+        return self.T % self.R == 0
+
+    def choose_keep(self, scores=None) -> list[int]:
+        """Indices (ascending) of the k = min(n, floor(r_d*T)) entries greatest in (score
+        descending, index ascending).  `scores` defaults to the accumulated scores; a parity test
+        may pass the kernel's own float32 scores to take the decision in the kernel's precision."""
+        n = len(self.Kd)
+        k = min(n, int(math.floor(self.r_d * self.T)))
+        sc = self.acc if scores is None else list(scores)
+        order = sorted(range(n), key=lambda j: (-sc[j], j))
+        return sorted(order[:k])
+
+    def apply_keep(self, kept: list[int]) -> list[int]:
+        """Compacts the decode region to the entries `kept` (ascending); returns the evicted ones."""
+        kept = sorted(int(j) for j in kept)
+        evicted = [j for j in range(len(self.Kd)) if j not in set(kept)]
+        self.Kd = [self.Kd[j] for j in kept]
+        self.Vd = [self.Vd[j] for j in kept]
+        self.acc = [self.acc[j] for j in kept]
+        self.born = [self.born[j] for j in kept]
         return evicted
+
+    def step(self, q: np.ndarray, k_new: np.ndarray, v_new: np.ndarray, decide_acc=None) -> list[int]:
+        """One generation step: accumulate, then every R steps keep the top floor(r_d*T) entries.
+        Returns the evicted indices (positions in the pre-eviction region)."""
+        self.accumulate(q, k_new, v_new)
+        if self.eviction_due():
+            return self.apply_keep(self.choose_keep(decide_acc))
+        return []
 
     @property
     def n_dec(self) -> int:

@@ -1,0 +1,662 @@
+// C ABI of the ShotKV hot path: argument validation, workspace carving and launch sequencing.
+// Every arithmetic step runs in the kernels of this directory; there is no host fallback.
+#include "../../include/shotkv.h"
+
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+#include "decode.cuh"
+#include "score_mma.cuh"
+#include "select_compact.cuh"
+
+using namespace shotkv;
+
+namespace {
+
+constexpr int kPieceMaxKeys = 512;     // longest key range one scoring work item covers
+constexpr int kMaxShots = 8192;
+constexpr int kStageSlots = 4;
+constexpr size_t kStageSlotBytes = 1u << 20;
+
+inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+struct shotkv_ctx {
+    int device = 0;
+    char err[512] = {0};
+    // pinned staging ring for the small host tables (offsets, piece lists) that go to the device
+    unsigned char* stage = nullptr;
+    cudaEvent_t stage_done[kStageSlots] = {};
+    int stage_next = 0;
+};
+
+namespace {
+
+int fail(shotkv_ctx* ctx, int code, const char* fmt, ...) {
+    if (ctx) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(ctx->err, sizeof(ctx->err), fmt, ap);
+        va_end(ap);
+    }
+    return code;
+}
+
+#define CUDA_TRY(ctx, expr)                                                                     \
+    do {                                                                                        \
+        cudaError_t e__ = (expr);                                                               \
+        if (e__ != cudaSuccess)                                                                 \
+            return fail(ctx, SHOTKV_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e__)); \
+    } while (0)
+
+int check_dims(const shotkv_dims* d, const char** why) {
+    if (!d) { *why = "dims is NULL"; return SHOTKV_ERR_INVALID_ARG; }
+    if (d->B < 1 || d->L < 1 || d->H < 1 || d->Hkv < 1 || d->N < 1 || d->W < 1 || d->S < 0) {
+        *why = "B, L, H, Hkv, N, W must be >= 1 and S >= 0"; return SHOTKV_ERR_INVALID_ARG;
+    }
+    if (d->H % d->Hkv != 0) { *why = "H must be a multiple of Hkv"; return SHOTKV_ERR_INVALID_ARG; }
+    if (d->W > d->N) { *why = "window W exceeds N"; return SHOTKV_ERR_INVALID_ARG; }
+    if (d->d != 64 && d->d != 128) { *why = "head dimension must be 64 or 128"; return SHOTKV_ERR_UNSUPPORTED_SHAPE; }
+    if ((long long)(d->H / d->Hkv) * d->W > 256) { *why = "G*W must be <= 256"; return SHOTKV_ERR_UNSUPPORTED_SHAPE; }
+    if (d->S > kMaxShots) { *why = "S must be <= 8192"; return SHOTKV_ERR_UNSUPPORTED_SHAPE; }
+    if ((long long)d->B * d->L * d->Hkv > 0x7fffffffLL / 256) { *why = "B*L*Hkv too large"; return SHOTKV_ERR_UNSUPPORTED_SHAPE; }
+    return SHOTKV_OK;
+}
+
+int check_policy_prefill(const shotkv_policy* p, const char** why) {
+    if (!p) { *why = "policy is NULL"; return SHOTKV_ERR_INVALID_ARG; }
+    if (!(p->r_p > 0.f) || !std::isfinite(p->r_p)) { *why = "r_p must be a positive finite number"; return SHOTKV_ERR_INVALID_ARG; }
+    if (p->select_mode != 0 && p->select_mode != 1) { *why = "select_mode must be 0 or 1"; return SHOTKV_ERR_INVALID_ARG; }
+    return SHOTKV_OK;
+}
+
+int budget_of(const shotkv_dims* d, const shotkv_policy* p) {
+    const double b = std::floor((double)p->r_p * (double)d->N);
+    return b > (double)d->N ? d->N : (int)b;
+}
+
+// 0 ok, negative error, or the warning; *max_always = largest always-kept count over the prompts
+int check_offsets(const shotkv_dims* d, const shotkv_policy* p, const int32_t* off, int* max_always, const char** why) {
+    if (!off) { *why = "offsets_host is NULL"; return SHOTKV_ERR_INVALID_ARG; }
+    int worst = 0;
+    for (int b = 0; b < d->B; ++b) {
+        const int32_t* o = off + (size_t)b * (d->S + 1);
+        if (o[0] < 0) { *why = "off[0] < 0"; return SHOTKV_ERR_BAD_OFFSETS; }
+        for (int i = 0; i < d->S; ++i)
+            if (o[i + 1] <= o[i]) { *why = "offsets must be strictly increasing (no empty shot)"; return SHOTKV_ERR_BAD_OFFSETS; }
+        if (o[d->S] > d->N - d->W) { *why = "off[S] > N - W: the window must lie after the last shot"; return SHOTKV_ERR_BAD_OFFSETS; }
+        const int always = o[0] + (d->N - o[d->S]);
+        if (always > worst) worst = always;
+    }
+    if (max_always) *max_always = worst;
+    if (p && worst > budget_of(d, p)) return SHOTKV_WARN_BUDGET_BELOW_ALWAYS_KEPT;
+    return SHOTKV_OK;
+}
+
+int rpad_of(const shotkv_dims* d) { return (d->H / d->Hkv) * d->W <= 128 ? 128 : 256; }
+int pmax_of(const shotkv_dims* d) { return d->S + 2 + d->N / kPieceMaxKeys + 1; }
+
+struct PrefillWs {
+    int* off;          // [B][S+1]
+    int2* pieces;      // [B][Pmax]
+    int* piece_seg;    // [B][Pmax]
+    float* part_m;     // [U][Pmax][Rpad]
+    float* part_z;
+    float* row_m;      // [U][Rpad]
+    float* row_invz;
+    float* unit_shot;  // [U][S]
+    size_t total;
+};
+
+PrefillWs carve(const shotkv_dims* d, void* base) {
+    PrefillWs w{};
+    const size_t U = (size_t)d->B * d->L * d->Hkv, P = pmax_of(d), R = rpad_of(d);
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o += align_up(bytes); return (unsigned char*)base + at; };
+    w.off = (int*)take((size_t)d->B * (d->S + 1) * 4);
+    w.pieces = (int2*)take((size_t)d->B * P * 8);
+    w.piece_seg = (int*)take((size_t)d->B * P * 4);
+    w.part_m = (float*)take(U * P * R * 4);
+    w.part_z = (float*)take(U * P * R * 4);
+    w.row_m = (float*)take(U * R * 4);
+    w.row_invz = (float*)take(U * R * 4);
+    w.unit_shot = (float*)take(U * (size_t)(d->S > 0 ? d->S : 1) * 4);
+    w.total = o;
+    return w;
+}
+
+// Copies `bytes` of host data to `dst` on `stream` through the context's pinned ring, so the
+// caller's buffer may be reused at once and the host does not wait for the stream.
+int upload_small(shotkv_ctx* ctx, void* dst, const void* src, size_t bytes, cudaStream_t stream) {
+    if (bytes == 0) return SHOTKV_OK;
+    if (bytes > kStageSlotBytes) {
+        CUDA_TRY(ctx, cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, stream));
+        CUDA_TRY(ctx, cudaStreamSynchronize(stream));
+        return SHOTKV_OK;
+    }
+    const int slot = ctx->stage_next;
+    ctx->stage_next = (slot + 1) % kStageSlots;
+    CUDA_TRY(ctx, cudaEventSynchronize(ctx->stage_done[slot]));
+    unsigned char* s = ctx->stage + (size_t)slot * kStageSlotBytes;
+    memcpy(s, src, bytes);
+    CUDA_TRY(ctx, cudaMemcpyAsync(dst, s, bytes, cudaMemcpyHostToDevice, stream));
+    CUDA_TRY(ctx, cudaEventRecord(ctx->stage_done[slot], stream));
+    return SHOTKV_OK;
+}
+
+// Splits [0, N) into pieces of at most kPieceMaxKeys keys.  With offsets: pieces never cross a
+// segment boundary (segment 0 = before the first shot, i+1 = shot i, S+1 = the question) and
+// piece_seg records the segment.  Without: plain fixed-size chunks.  Returns pieces per prompt
+// (padded with empty pieces to the same count for every prompt).
+int build_pieces(const shotkv_dims* d, const int32_t* off, std::vector<int2>& pieces, std::vector<int>& seg) {
+    std::vector<std::vector<int2>> pp(d->B);
+    std::vector<std::vector<int>> ss(d->B);
+    size_t P = 0;
+    for (int b = 0; b < d->B; ++b) {
+        auto add_range = [&](int lo, int hi, int s) {
+            for (int x = lo; x < hi; x += kPieceMaxKeys) {
+                pp[b].push_back(make_int2(x, x + kPieceMaxKeys < hi ? x + kPieceMaxKeys : hi));
+                ss[b].push_back(s);
+            }
+        };
+        if (off) {
+            const int32_t* o = off + (size_t)b * (d->S + 1);
+            add_range(0, o[0], 0);
+            for (int i = 0; i < d->S; ++i) add_range(o[i], o[i + 1], i + 1);
+            add_range(o[d->S], d->N, d->S + 1);
+        } else {
+            add_range(0, d->N, 0);
+        }
+        if (pp[b].size() > P) P = pp[b].size();
+    }
+    pieces.assign((size_t)d->B * P, make_int2(0, 0));
+    seg.assign((size_t)d->B * P, d->S + 2);
+    for (int b = 0; b < d->B; ++b)
+        for (size_t i = 0; i < pp[b].size(); ++i) {
+            pieces[(size_t)b * P + i] = pp[b][i];
+            seg[(size_t)b * P + i] = ss[b][i];
+        }
+    return (int)P;
+}
+
+template <int D, int MB, bool COLSUM>
+int launch_score_t(shotkv_ctx* ctx, const ScoreParams& sp, int U, cudaStream_t stream) {
+    constexpr int smem = score_mma_smem_bytes<D, MB>();
+    static bool attr_done[64] = {};
+    int dev = ctx->device;
+    if (dev < 64 && !attr_done[dev]) {
+        CUDA_TRY(ctx, cudaFuncSetAttribute(score_mma_kernel<D, MB, COLSUM>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        attr_done[dev] = true;
+    } else if (dev >= 64) {
+        CUDA_TRY(ctx, cudaFuncSetAttribute(score_mma_kernel<D, MB, COLSUM>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    }
+    dim3 grid((sp.P + sp.ppc - 1) / sp.ppc, U);
+    score_mma_kernel<D, MB, COLSUM><<<grid, 256, smem, stream>>>(sp);
+    CUDA_TRY(ctx, cudaGetLastError());
+    return SHOTKV_OK;
+}
+
+template <bool COLSUM>
+int launch_score(shotkv_ctx* ctx, const shotkv_dims* d, const ScoreParams& sp, int U, cudaStream_t stream) {
+    const bool big = sp.Rpad == 256;
+    if (d->d == 128) return big ? launch_score_t<128, 2, COLSUM>(ctx, sp, U, stream) : launch_score_t<128, 1, COLSUM>(ctx, sp, U, stream);
+    return big ? launch_score_t<64, 2, COLSUM>(ctx, sp, U, stream) : launch_score_t<64, 1, COLSUM>(ctx, sp, U, stream);
+}
+
+ScoreParams base_params(const shotkv_dims* d, const shotkv_bf16* Q, const shotkv_bf16* K, const PrefillWs& w, int P) {
+    ScoreParams sp{};
+    sp.Q = reinterpret_cast<const __nv_bfloat16*>(Q);
+    sp.K = reinterpret_cast<const __nv_bfloat16*>(K);
+    sp.pieces = w.pieces;
+    sp.P = P;
+    const long long U = (long long)d->B * d->L * d->Hkv;
+    int ppc = (int)((U * P) / (148 * 8));     // aim for >= 8 work items per SM
+    sp.ppc = ppc < 1 ? 1 : (ppc > 8 ? 8 : ppc);
+    sp.L = d->L; sp.H = d->H; sp.Hkv = d->Hkv; sp.N = d->N; sp.W = d->W;
+    sp.G = d->H / d->Hkv; sp.R = sp.G * d->W; sp.Rpad = rpad_of(d);
+    sp.scale_log2 = kLog2e / sqrtf((float)d->d);
+    sp.part_m = w.part_m; sp.part_z = w.part_z;
+    sp.row_m = w.row_m; sp.row_invz = w.row_invz;
+    sp.imp = nullptr;
+    return sp;
+}
+
+int set_device(shotkv_ctx* ctx) {
+    if (!ctx) return SHOTKV_ERR_INVALID_ARG;
+    CUDA_TRY(ctx, cudaSetDevice(ctx->device));
+    return SHOTKV_OK;
+}
+
+int check_ws(shotkv_ctx* ctx, const shotkv_dims* d, void* ws, size_t ws_bytes) {
+    if (!ws) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "workspace is NULL");
+    if ((uintptr_t)ws % 256) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
+    const size_t need = shotkv_workspace_bytes(d);
+    if (ws_bytes < need) return fail(ctx, SHOTKV_ERR_WORKSPACE_TOO_SMALL, "workspace has %zu bytes, %zu needed", ws_bytes, need);
+    return SHOTKV_OK;
+}
+
+// STATS pass over `pieces` followed by the per-row reduction; leaves part_m/part_z (and for the
+// token path row_m/row_invz) in the workspace.
+int run_stats(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const shotkv_bf16* K, const PrefillWs& w,
+              const int32_t* off_host, bool need_rows, int* P_out, cudaStream_t stream) {
+    std::vector<int2> pieces;
+    std::vector<int> seg;
+    const int P = build_pieces(d, off_host, pieces, seg);
+    if (P > pmax_of(d)) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "internal: piece count %d exceeds bound %d", P, pmax_of(d));
+    int rc = upload_small(ctx, w.pieces, pieces.data(), pieces.size() * sizeof(int2), stream);
+    if (rc) return rc;
+    rc = upload_small(ctx, w.piece_seg, seg.data(), seg.size() * sizeof(int), stream);
+    if (rc) return rc;
+    const int U = d->B * d->L * d->Hkv;
+    ScoreParams sp = base_params(d, Q, K, w, P);
+    rc = launch_score<false>(ctx, d, sp, U, stream);
+    if (rc) return rc;
+    if (need_rows) {
+        row_stats_kernel<<<U, 256, 0, stream>>>(w.part_m, w.part_z, P, sp.R, sp.Rpad, w.row_m, w.row_invz);
+        CUDA_TRY(ctx, cudaGetLastError());
+    }
+    *P_out = P;
+    return SHOTKV_OK;
+}
+
+int run_select(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_policy* p, const PrefillWs& w, float* shot_scores,
+               uint8_t* keep, int32_t* kept_idx, int32_t* kept_count, int32_t Mcap, cudaStream_t stream) {
+    const size_t smem = (size_t)d->S * 16 + (kSelectThreads + 1) * 4 + 16;
+    static bool attr_done = false;
+    if (smem > 48 * 1024 || !attr_done) {
+        CUDA_TRY(ctx, cudaFuncSetAttribute(select_shots_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
+        attr_done = true;
+    }
+    select_shots_kernel<<<d->B * d->L, kSelectThreads, smem, stream>>>(shot_scores, w.off, d->L, d->N, d->S, budget_of(d, p),
+                                                                     p->select_mode, Mcap, keep, kept_idx, kept_count);
+    CUDA_TRY(ctx, cudaGetLastError());
+    return SHOTKV_OK;
+}
+
+int run_compact(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* K, const shotkv_bf16* V, const int32_t* kept_idx,
+                const int32_t* kept_count, int32_t Mcap, shotkv_bf16* Kc, shotkv_bf16* Vc, cudaStream_t stream) {
+    const int rows_per_cta = d->d == 128 ? 64 : 128;
+    int gx = (Mcap + rows_per_cta - 1) / rows_per_cta;
+    if (gx < 1) gx = 1;
+    dim3 grid(gx, d->Hkv, d->B * d->L);
+    if (grid.z > 65535) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "B*L must be <= 65535");
+    if (d->d == 128)
+        compact_kv_kernel<128><<<grid, 256, 0, stream>>>((const uint4*)K, (const uint4*)V, kept_idx, kept_count, d->Hkv, d->N, Mcap, (uint4*)Kc, (uint4*)Vc);
+    else
+        compact_kv_kernel<64><<<grid, 256, 0, stream>>>((const uint4*)K, (const uint4*)V, kept_idx, kept_count, d->Hkv, d->N, Mcap, (uint4*)Kc, (uint4*)Vc);
+    CUDA_TRY(ctx, cudaGetLastError());
+    return SHOTKV_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------
+extern "C" {
+
+const char* shotkv_version(void) { return "shotkv-b200 0.1"; }
+
+int shotkv_create(shotkv_ctx** out, int device) {
+    if (!out) return SHOTKV_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return SHOTKV_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return SHOTKV_ERR_CUDA;
+    if (prop.major != 10) return SHOTKV_ERR_CUDA;   // built for sm_100a only
+    if (cudaSetDevice(device) != cudaSuccess) return SHOTKV_ERR_CUDA;
+    shotkv_ctx* ctx = new (std::nothrow) shotkv_ctx;
+    if (!ctx) return SHOTKV_ERR_INVALID_ARG;
+    ctx->device = device;
+    if (cudaMallocHost((void**)&ctx->stage, kStageSlots * kStageSlotBytes) != cudaSuccess) {
+        delete ctx;
+        return SHOTKV_ERR_CUDA;
+    }
+    for (int i = 0; i < kStageSlots; ++i)
+        if (cudaEventCreateWithFlags(&ctx->stage_done[i], cudaEventDisableTiming) != cudaSuccess) {
+            cudaFreeHost(ctx->stage);
+            delete ctx;
+            return SHOTKV_ERR_CUDA;
+        }
+    *out = ctx;
+    return SHOTKV_OK;
+}
+
+void shotkv_destroy(shotkv_ctx* ctx) {
+    if (!ctx) return;
+    cudaSetDevice(ctx->device);
+    for (int i = 0; i < kStageSlots; ++i)
+        if (ctx->stage_done[i]) {
+            cudaEventSynchronize(ctx->stage_done[i]);
+            cudaEventDestroy(ctx->stage_done[i]);
+        }
+    if (ctx->stage) cudaFreeHost(ctx->stage);
+    delete ctx;
+}
+
+const char* shotkv_last_error(const shotkv_ctx* ctx) { return ctx ? ctx->err : "context is NULL"; }
+
+int32_t shotkv_budget_tokens(const shotkv_dims* dims, const shotkv_policy* policy) {
+    const char* why = "";
+    if (check_dims(dims, &why) || check_policy_prefill(policy, &why)) return SHOTKV_ERR_INVALID_ARG;
+    return budget_of(dims, policy);
+}
+
+int32_t shotkv_kept_capacity(const shotkv_dims* dims, const shotkv_policy* policy, const int32_t* offsets_host) {
+    const char* why = "";
+    int rc = check_dims(dims, &why);
+    if (rc) return rc;
+    rc = check_policy_prefill(policy, &why);
+    if (rc) return rc;
+    int worst = 0;
+    rc = check_offsets(dims, policy, offsets_host, &worst, &why);
+    if (rc < 0) return rc;
+    const int b = budget_of(dims, policy);
+    return b > worst ? b : worst;
+}
+
+int shotkv_validate(const shotkv_dims* dims, const shotkv_policy* policy, const int32_t* offsets_host) {
+    const char* why = "";
+    int rc = check_dims(dims, &why);
+    if (rc) return rc;
+    if (policy) {
+        rc = check_policy_prefill(policy, &why);
+        if (rc) return rc;
+    }
+    if (offsets_host) return check_offsets(dims, policy, offsets_host, nullptr, &why);
+    return SHOTKV_OK;
+}
+
+size_t shotkv_workspace_bytes(const shotkv_dims* dims) {
+    const char* why = "";
+    if (check_dims(dims, &why)) return 0;
+    return carve(dims, nullptr).total;
+}
+
+int shotkv_prefill_score(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_bf16* Qwin, const shotkv_bf16* K,
+                         float* token_importance, void* ws, size_t ws_bytes, void* stream_) {
+    int rc = set_device(ctx);
+    if (rc) return rc;
+    const char* why = "";
+    if ((rc = check_dims(dims, &why))) return fail(ctx, rc, "%s", why);
+    if (!Qwin || !K || !token_importance) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "Qwin, K and token_importance must not be NULL");
+    if ((rc = check_ws(ctx, dims, ws, ws_bytes))) return rc;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    const PrefillWs w = carve(dims, ws);
+    int P = 0;
+    if ((rc = run_stats(ctx, dims, Qwin, K, w, nullptr, true, &P, stream))) return rc;
+    ScoreParams sp = base_params(dims, Qwin, K, w, P);
+    sp.imp = token_importance;
+    return launch_score<true>(ctx, dims, sp, dims->B * dims->L * dims->Hkv, stream);
+}
+
+int shotkv_select_shots(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_policy* policy,
+                        const float* token_importance, const int32_t* offsets_host, float* shot_scores, uint8_t* keep,
+                        int32_t* kept_idx, int32_t* kept_count, int32_t Mcap, void* ws, size_t ws_bytes, void* stream_) {
+    int rc = set_device(ctx);
+    if (rc) return rc;
+    const char* why = "";
+    if ((rc = check_dims(dims, &why))) return fail(ctx, rc, "%s", why);
+    if ((rc = check_policy_prefill(policy, &why))) return fail(ctx, rc, "%s", why);
+    int worst = 0;
+    const int orc = check_offsets(dims, policy, offsets_host, &worst, &why);
+    if (orc < 0) return fail(ctx, orc, "%s", why);
+    if (!shot_scores || !keep || !kept_idx || !kept_count) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "output pointers must not be NULL");
+    const int need = budget_of(dims, policy) > worst ? budget_of(dims, policy) : worst;
+    if (Mcap < need) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "Mcap = %d but %d rows may be kept", Mcap, need);
+    if ((rc = check_ws(ctx, dims, ws, ws_bytes))) return rc;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    const PrefillWs w = carve(dims, ws);
+    if ((rc = upload_small(ctx, w.off, offsets_host, (size_t)dims->B * (dims->S + 1) * 4, stream))) return rc;
+    if (token_importance && dims->S > 0) {
+        dim3 grid(dims->S, dims->B * dims->L);
+        shot_score_from_tokens_kernel<<<grid, 128, 0, stream>>>(token_importance, w.off, dims->L, dims->Hkv, dims->N, dims->S, shot_scores);
+        CUDA_TRY(ctx, cudaGetLastError());
+    }
+    if ((rc = run_select(ctx, dims, policy, w, shot_scores, keep, kept_idx, kept_count, Mcap, stream))) return rc;
+    if (orc > 0) fail(ctx, orc, "always-kept tokens (%d) exceed the budget (%d) for some prompt", worst, budget_of(dims, policy));
+    return orc;
+}
+
+int shotkv_compact_kv(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_bf16* K, const shotkv_bf16* V,
+                      const int32_t* kept_idx, const int32_t* kept_count, int32_t Mcap, shotkv_bf16* Kc, shotkv_bf16* Vc,
+                      void* stream_) {
+    int rc = set_device(ctx);
+    if (rc) return rc;
+    const char* why = "";
+    if ((rc = check_dims(dims, &why))) return fail(ctx, rc, "%s", why);
+    if (!K || !V || !kept_idx || !kept_count || !Kc || !Vc) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "pointers must not be NULL");
+    if (Mcap < 1) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "Mcap must be >= 1");
+    return run_compact(ctx, dims, K, V, kept_idx, kept_count, Mcap, Kc, Vc, (cudaStream_t)stream_);
+}
+
+int shotkv_prefill_compress(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_policy* policy, const shotkv_bf16* Qwin,
+                            const shotkv_bf16* K, const shotkv_bf16* V, const int32_t* offsets_host, float* shot_scores,
+                            uint8_t* keep, int32_t* kept_idx, int32_t* kept_count, int32_t Mcap, shotkv_bf16* Kc,
+                            shotkv_bf16* Vc, float* token_importance, uint32_t flags, void* ws, size_t ws_bytes,
+                            void* stream_) {
+    int rc = set_device(ctx);
+    if (rc) return rc;
+    if (flags & SHOTKV_FLAG_TOKEN_IMPORTANCE) {
+        if ((rc = shotkv_prefill_score(ctx, dims, Qwin, K, token_importance, ws, ws_bytes, stream_)) < 0) return rc;
+        const int src = shotkv_select_shots(ctx, dims, policy, token_importance, offsets_host, shot_scores, keep, kept_idx,
+                                            kept_count, Mcap, ws, ws_bytes, stream_);
+        if (src < 0) return src;
+        if ((rc = shotkv_compact_kv(ctx, dims, K, V, kept_idx, kept_count, Mcap, Kc, Vc, stream_)) < 0) return rc;
+        return src;
+    }
+    const char* why = "";
+    if ((rc = check_dims(dims, &why))) return fail(ctx, rc, "%s", why);
+    if ((rc = check_policy_prefill(policy, &why))) return fail(ctx, rc, "%s", why);
+    int worst = 0;
+    const int orc = check_offsets(dims, policy, offsets_host, &worst, &why);
+    if (orc < 0) return fail(ctx, orc, "%s", why);
+    if (!Qwin || !K || !V || !shot_scores || !keep || !kept_idx || !kept_count || !Kc || !Vc)
+        return fail(ctx, SHOTKV_ERR_INVALID_ARG, "pointers must not be NULL");
+    const int need = budget_of(dims, policy) > worst ? budget_of(dims, policy) : worst;
+    if (Mcap < need) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "Mcap = %d but %d rows may be kept", Mcap, need);
+    if ((rc = check_ws(ctx, dims, ws, ws_bytes))) return rc;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    const PrefillWs w = carve(dims, ws);
+    if ((rc = upload_small(ctx, w.off, offsets_host, (size_t)dims->B * (dims->S + 1) * 4, stream))) return rc;
+    int P = 0;
+    if ((rc = run_stats(ctx, dims, Qwin, K, w, offsets_host, false, &P, stream))) return rc;
+    const int U = dims->B * dims->L * dims->Hkv;
+    const int R = (dims->H / dims->Hkv) * dims->W, Rpad = rpad_of(dims);
+    if (dims->S > 0) {
+        if (Rpad == 128)
+            shot_mass_kernel<128><<<U, 128, 0, stream>>>(w.part_m, w.part_z, w.piece_seg, P, R, Rpad, dims->L, dims->Hkv, dims->S, w.unit_shot);
+        else
+            shot_mass_kernel<256><<<U, 256, 0, stream>>>(w.part_m, w.part_z, w.piece_seg, P, R, Rpad, dims->L, dims->Hkv, dims->S, w.unit_shot);
+        CUDA_TRY(ctx, cudaGetLastError());
+        shot_score_from_mass_kernel<<<dims->B * dims->L, 128, 0, stream>>>(w.unit_shot, w.off, dims->L, dims->Hkv, dims->S, shot_scores);
+        CUDA_TRY(ctx, cudaGetLastError());
+    }
+    if ((rc = run_select(ctx, dims, policy, w, shot_scores, keep, kept_idx, kept_count, Mcap, stream))) return rc;
+    if ((rc = run_compact(ctx, dims, K, V, kept_idx, kept_count, Mcap, Kc, Vc, stream))) return rc;
+    if (orc > 0) fail(ctx, orc, "always-kept tokens (%d) exceed the budget (%d) for some prompt", worst, budget_of(dims, policy));
+    return orc;
+}
+
+// ---- host-buffer variant -------------------------------------------------------------------
+namespace {
+struct HostArena {
+    shotkv_bf16 *Q, *K, *V, *Kc, *Vc;
+    float* scores;
+    uint8_t* keep;
+    int32_t *idx, *count;
+    void* ws;
+    size_t ws_bytes, total;
+};
+HostArena carve_host(const shotkv_dims* d, int32_t Mcap, void* base) {
+    HostArena a{};
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o += align_up(bytes); return (unsigned char*)base + at; };
+    const size_t BL = (size_t)d->B * d->L, U = BL * d->Hkv;
+    a.Q = (shotkv_bf16*)take(BL * d->H * d->W * d->d * 2);
+    a.K = (shotkv_bf16*)take(U * d->N * d->d * 2);
+    a.V = (shotkv_bf16*)take(U * d->N * d->d * 2);
+    a.Kc = (shotkv_bf16*)take(U * (size_t)Mcap * d->d * 2);
+    a.Vc = (shotkv_bf16*)take(U * (size_t)Mcap * d->d * 2);
+    a.scores = (float*)take(BL * (size_t)(d->S > 0 ? d->S : 1) * 4);
+    a.keep = (uint8_t*)take(BL * (size_t)(d->S > 0 ? d->S : 1));
+    a.idx = (int32_t*)take(BL * (size_t)Mcap * 4);
+    a.count = (int32_t*)take(BL * 4);
+    a.ws_bytes = shotkv_workspace_bytes(d);
+    a.ws = take(a.ws_bytes);
+    a.total = o;
+    return a;
+}
+}  // namespace
+
+size_t shotkv_host_arena_bytes(const shotkv_dims* dims, int32_t Mcap) {
+    const char* why = "";
+    if (check_dims(dims, &why) || Mcap < 1) return 0;
+    return carve_host(dims, Mcap, nullptr).total;
+}
+
+int shotkv_prefill_compress_host(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_policy* policy,
+                                 const shotkv_bf16* Qwin_host, const shotkv_bf16* K_host, const shotkv_bf16* V_host,
+                                 const int32_t* offsets_host, float* shot_scores_host, uint8_t* keep_host,
+                                 int32_t* kept_idx_host, int32_t* kept_count_host, int32_t Mcap, shotkv_bf16* Kc_host,
+                                 shotkv_bf16* Vc_host, void* arena, size_t arena_bytes, void* stream_) {
+    int rc = set_device(ctx);
+    if (rc) return rc;
+    const char* why = "";
+    if ((rc = check_dims(dims, &why))) return fail(ctx, rc, "%s", why);
+    if (!Qwin_host || !K_host || !V_host) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "host inputs must not be NULL");
+    if (Mcap < 1) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "Mcap must be >= 1");
+    if (!arena || (uintptr_t)arena % 256) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "arena must be a 256-byte aligned device buffer");
+    const HostArena a = carve_host(dims, Mcap, arena);
+    if (arena_bytes < a.total) return fail(ctx, SHOTKV_ERR_WORKSPACE_TOO_SMALL, "arena has %zu bytes, %zu needed", arena_bytes, a.total);
+    cudaStream_t stream = (cudaStream_t)stream_;
+    const size_t BL = (size_t)dims->B * dims->L, U = BL * dims->Hkv;
+    CUDA_TRY(ctx, cudaMemcpyAsync(a.Q, Qwin_host, BL * dims->H * dims->W * dims->d * 2, cudaMemcpyHostToDevice, stream));
+    CUDA_TRY(ctx, cudaMemcpyAsync(a.K, K_host, U * dims->N * dims->d * 2, cudaMemcpyHostToDevice, stream));
+    CUDA_TRY(ctx, cudaMemcpyAsync(a.V, V_host, U * dims->N * dims->d * 2, cudaMemcpyHostToDevice, stream));
+    const int prc = shotkv_prefill_compress(ctx, dims, policy, a.Q, a.K, a.V, offsets_host, a.scores, a.keep, a.idx, a.count,
+                                            Mcap, a.Kc, a.Vc, nullptr, 0, a.ws, a.ws_bytes, stream_);
+    if (prc < 0) return prc;
+    const size_t S1 = dims->S > 0 ? dims->S : 1;
+    if (shot_scores_host) CUDA_TRY(ctx, cudaMemcpyAsync(shot_scores_host, a.scores, BL * S1 * 4, cudaMemcpyDeviceToHost, stream));
+    if (keep_host) CUDA_TRY(ctx, cudaMemcpyAsync(keep_host, a.keep, BL * S1, cudaMemcpyDeviceToHost, stream));
+    if (kept_idx_host) CUDA_TRY(ctx, cudaMemcpyAsync(kept_idx_host, a.idx, BL * (size_t)Mcap * 4, cudaMemcpyDeviceToHost, stream));
+    if (kept_count_host) CUDA_TRY(ctx, cudaMemcpyAsync(kept_count_host, a.count, BL * 4, cudaMemcpyDeviceToHost, stream));
+    if (Kc_host) CUDA_TRY(ctx, cudaMemcpyAsync(Kc_host, a.Kc, U * (size_t)Mcap * dims->d * 2, cudaMemcpyDeviceToHost, stream));
+    if (Vc_host) CUDA_TRY(ctx, cudaMemcpyAsync(Vc_host, a.Vc, U * (size_t)Mcap * dims->d * 2, cudaMemcpyDeviceToHost, stream));
+    return prc;
+}
+
+// ---- decode ---------------------------------------------------------------------------------
+size_t shotkv_decode_workspace_bytes(const shotkv_dims* dims, int32_t Dcap) {
+    if (!dims || Dcap < 1 || dims->B < 1 || dims->L < 1 || dims->Hkv < 1) return 0;
+    const size_t BL = (size_t)dims->B * dims->L;
+    return align_up(BL * dims->Hkv * (size_t)Dcap * 4) + align_up(BL * (size_t)Dcap * 4);
+}
+
+int32_t shotkv_decode_capacity(const shotkv_policy* policy, int32_t steps) {
+    if (!policy || steps < 0 || policy->recompress_every < 1 || !(policy->r_d >= 0.f)) return SHOTKV_ERR_INVALID_ARG;
+    // replay the host-side counters
+    int n = 0, worst = 1;
+    for (int T = 1; T <= steps; ++T) {
+        ++n;
+        if (n > worst) worst = n;
+        if (T % policy->recompress_every == 0) {
+            const int k = (int)std::floor((double)policy->r_d * (double)T);
+            if (k < n) n = k;
+        }
+    }
+    return worst;
+}
+
+int shotkv_decode_init(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_policy* policy, int32_t Dcap, int32_t Mcap,
+                       shotkv_bf16* Kd, shotkv_bf16* Vd, float* acc, int32_t* born, void* ws, size_t ws_bytes,
+                       shotkv_decode_state* state) {
+    if (!ctx) return SHOTKV_ERR_INVALID_ARG;
+    if (!dims || !policy || !state) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "dims, policy and state must not be NULL");
+    if (dims->B < 1 || dims->L < 1 || dims->H < 1 || dims->Hkv < 1 || dims->H % dims->Hkv)
+        return fail(ctx, SHOTKV_ERR_INVALID_ARG, "B, L, H, Hkv must be >= 1 and H a multiple of Hkv");
+    if (dims->d != 64 && dims->d != 128) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "head dimension must be 64 or 128");
+    if (dims->H / dims->Hkv > 8) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "decode supports H/Hkv <= 8");
+    if (!(policy->r_d >= 0.f) || !std::isfinite(policy->r_d)) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "r_d must be finite and >= 0");
+    if (policy->recompress_every < 1) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "recompress_every must be >= 1");
+    if (policy->protect_recent != 0) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "protect_recent must be 0");
+    if (Dcap < 1 || Dcap > 4096) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "Dcap must be in [1, 4096]");
+    if (Mcap < 0) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "Mcap must be >= 0");
+    if (!Kd || !Vd || !acc || !born || !ws) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "device pointers must not be NULL");
+    if (ws_bytes < shotkv_decode_workspace_bytes(dims, Dcap))
+        return fail(ctx, SHOTKV_ERR_WORKSPACE_TOO_SMALL, "decode workspace has %zu bytes, %zu needed", ws_bytes,
+                    shotkv_decode_workspace_bytes(dims, Dcap));
+    memset(state, 0, sizeof(*state));
+    state->dims = *dims;
+    state->policy = *policy;
+    state->Dcap = Dcap;
+    state->Mcap = Mcap;
+    state->Kd = Kd; state->Vd = Vd; state->acc = acc; state->born = born;
+    state->ws = ws; state->ws_bytes = ws_bytes;
+    return SHOTKV_OK;
+}
+
+int shotkv_decode_step(shotkv_ctx* ctx, shotkv_decode_state* st, const shotkv_bf16* q, const shotkv_bf16* k_new,
+                       const shotkv_bf16* v_new, const shotkv_bf16* Kc, const int32_t* kept_count, void* stream_) {
+    int rc = set_device(ctx);
+    if (rc) return rc;
+    if (!st || !q || !k_new || !v_new || !kept_count) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "pointers must not be NULL");
+    if (st->Mcap > 0 && !Kc) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "Kc must not be NULL when Mcap > 0");
+    if (st->n_dec + 1 > st->Dcap) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "decode region full: n_dec = %d, Dcap = %d", st->n_dec, st->Dcap);
+    cudaStream_t stream = (cudaStream_t)stream_;
+    const shotkv_dims& d = st->dims;
+    const int BL = d.B * d.L, U = BL * d.Hkv;
+    float* partial = (float*)st->ws;
+    int* keep_pos = (int*)((unsigned char*)st->ws + align_up((size_t)U * st->Dcap * 4));
+
+    DecodeParams p{};
+    p.q = (const __nv_bfloat16*)q; p.k_new = (const __nv_bfloat16*)k_new; p.v_new = (const __nv_bfloat16*)v_new;
+    p.Kc = (const __nv_bfloat16*)Kc; p.kept_count = kept_count;
+    p.Kd = (__nv_bfloat16*)st->Kd; p.Vd = (__nv_bfloat16*)st->Vd; p.partial = partial;
+    p.H = d.H; p.Hkv = d.Hkv; p.G = d.H / d.Hkv; p.Mcap = st->Mcap; p.Dcap = st->Dcap; p.n_old = st->n_dec;
+    p.scale_log2 = kLog2e / sqrtf((float)d.d);
+    const size_t smem = (size_t)8 * st->Dcap * 4 + (8 * 8 * 2 + 16) * 4;
+    if (d.d == 128) {
+        CUDA_TRY(ctx, cudaFuncSetAttribute(decode_score_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        decode_score_kernel<128><<<U, 256, smem, stream>>>(p);
+    } else {
+        CUDA_TRY(ctx, cudaFuncSetAttribute(decode_score_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        decode_score_kernel<64><<<U, 256, smem, stream>>>(p);
+    }
+    CUDA_TRY(ctx, cudaGetLastError());
+    decode_accumulate_kernel<<<BL, 128, 0, stream>>>(partial, d.Hkv, st->Dcap, st->n_dec, st->T, st->acc, st->born);
+    CUDA_TRY(ctx, cudaGetLastError());
+    st->n_dec += 1;
+    st->T += 1;
+    if (st->T % st->policy.recompress_every == 0) {
+        const int n = st->n_dec;
+        int k = (int)std::floor((double)st->policy.r_d * (double)st->T);
+        if (k > n) k = n;
+        if (k < n) {
+            const size_t rs = (size_t)n * 16 + (kSelectThreads + 1) * 4 + 16;
+            CUDA_TRY(ctx, cudaFuncSetAttribute(decode_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
+            decode_rank_kernel<<<BL, kSelectThreads, rs, stream>>>(st->acc, st->born, st->Dcap, n, k, keep_pos);
+            CUDA_TRY(ctx, cudaGetLastError());
+            if (k > 0) {
+                dim3 grid(U, 2);
+                if (d.d == 128)
+                    decode_compact_kernel<128><<<grid, 256, 0, stream>>>((__nv_bfloat16*)st->Kd, (__nv_bfloat16*)st->Vd, keep_pos, d.Hkv, st->Dcap, k);
+                else
+                    decode_compact_kernel<64><<<grid, 256, 0, stream>>>((__nv_bfloat16*)st->Kd, (__nv_bfloat16*)st->Vd, keep_pos, d.Hkv, st->Dcap, k);
+                CUDA_TRY(ctx, cudaGetLastError());
+            }
+            st->n_dec = k;
+        }
+    }
+    return SHOTKV_OK;
+}
+
+}  // extern "C"

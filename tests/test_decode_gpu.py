@@ -1,0 +1,141 @@
+"""GPU parity tests of Phase 2 (per-step score accumulation, periodic top-k eviction) against
+the CPU oracle run in lock-step on the same bytes."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2502_01941_b200 as skv
+from oracle import shotkv_oracle as O
+from paper_2502_01941_b200 import workloads as wl
+import parity as P
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2502_01941_b200.build import build_library
+    build_library()
+    c = skv.Context(0)
+    yield c
+    c.close()
+
+
+class GpuDecoder:
+    def __init__(self, ctx, cfg: wl.DecodeConfig, Kc, kept_count, Dcap=None):
+        self.ctx, self.cfg = ctx, cfg
+        self.dims = skv.make_dims(cfg.B, cfg.L, cfg.H, cfg.Hkv, cfg.d, 1, 1, 0)
+        self.pol = skv.make_policy(r_d=cfg.r_d, recompress_every=cfg.recompress_every)
+        self.Dcap = Dcap or skv.shotkv_decode_capacity(self.pol, cfg.steps)
+        dev = "cuda"
+        self.Kd = torch.zeros(cfg.B, cfg.L, cfg.Hkv, self.Dcap, cfg.d, dtype=torch.bfloat16, device=dev)
+        self.Vd = torch.zeros_like(self.Kd)
+        self.acc = torch.zeros(cfg.B, cfg.L, self.Dcap, dtype=torch.float32, device=dev)
+        self.born = torch.full((cfg.B, cfg.L, self.Dcap), -1, dtype=torch.int32, device=dev)
+        self.ws = torch.empty(skv.shotkv_decode_workspace_bytes(self.dims, self.Dcap), dtype=torch.uint8, device=dev)
+        self.Kc, self.kept_count = Kc, kept_count
+        self.state = skv.shotkv_decode_init(ctx, self.dims, self.pol, self.Dcap, Kc.shape[3], self.Kd, self.Vd, self.acc,
+                                            self.born, self.ws)
+
+    def step(self, q, k, v):
+        skv.shotkv_decode_step(self.ctx, self.state, q, k, v, self.Kc, self.kept_count)
+
+
+def lockstep(ctx, cfg, M, units, counts=None, steps=None):
+    """Runs `steps` decode steps on the GPU for the whole batch and the oracle for `units`,
+    comparing after every step.  Returns the number of reported eviction ties."""
+    Kc, kept = wl.random_prefill_cache(cfg, M, "cuda", counts)
+    gpu = GpuDecoder(ctx, cfg, Kc, kept)
+    orc = {}
+    for (b, l) in units:
+        m = int(kept[b, l])
+        orc[(b, l)] = O.DecodeOracle(wl.bf16_to_f64(Kc[b, l, :, :m]), cfg.H, cfg.r_d, cfg.recompress_every)
+    ties = 0
+    for s in range(steps or cfg.steps):
+        q, k, v = wl.decode_step_inputs(cfg, s, "cuda")
+        gpu.step(q, k, v)
+        torch.cuda.synchronize()
+        n = gpu.state.n_dec
+        assert gpu.state.T == s + 1
+        g_born = gpu.born.cpu().numpy()
+        g_acc = gpu.acc.cpu().numpy()
+        for (b, l), o in orc.items():
+            o.accumulate(wl.bf16_to_f64(q[b, l]), wl.bf16_to_f64(k[b, l]), wl.bf16_bits(v[b, l]))
+            if o.eviction_due():
+                want = o.choose_keep()
+                got_born = g_born[b, l, :n].tolist()
+                got = [o.born.index(t) for t in got_born]        # GPU's survivors as oracle indices
+                if got != want:
+                    # accepted only as a near-tie at the cut: every entry in one set but not the
+                    # other has an oracle score within the tolerance of the cut score
+                    diff = set(got) ^ set(want)
+                    sc = np.array(o.acc)
+                    cut = min(sc[j] for j in want) if want else 0.0
+                    for j in diff:
+                        assert abs(sc[j] - cut) <= 2 * (P.SCORE_RTOL * abs(cut) + P.SCORE_ATOL), \
+                            f"step {s}: eviction differs beyond a tie"
+                    ties += 1
+                    want = sorted(got)
+                o.apply_keep(want)
+            assert o.n_dec == n and o.born == g_born[b, l, :n].tolist()
+            ref = np.array(o.acc)
+            err = np.abs(g_acc[b, l, :n] - ref)
+            assert np.all(err <= P.SCORE_RTOL * np.abs(ref) + P.SCORE_ATOL), f"step {s}: acc off by {err.max()}"
+            # the decode region itself: bit-exact keys and values in position order
+            if (s + 1) % cfg.recompress_every == 0 or s < 3:
+                kd = wl.bf16_to_f64(gpu.Kd[b, l, :, :n])
+                np.testing.assert_array_equal(kd, np.stack(o.Kd, axis=1)) if n else None
+                vd = wl.bf16_bits(gpu.Vd[b, l, :, :n])
+                np.testing.assert_array_equal(vd, np.stack(o.Vd, axis=1)) if n else None
+    return ties
+
+
+def test_decode_small_lockstep(ctx):
+    cfg = wl.DecodeConfig("dec_small", B=2, L=2, H=8, Hkv=2, d=128, steps=70, r_d=0.25, recompress_every=8, cfg_id=21)
+    counts = np.array([[100, 37], [64, 1]], np.int32)
+    ties = lockstep(ctx, cfg, 100, [(0, 0), (0, 1), (1, 0), (1, 1)], counts)
+    assert ties <= 2
+
+
+def test_decode_d64_every_step_and_keep_all(ctx):
+    cfg = wl.DecodeConfig("dec_d64", B=1, L=2, H=4, Hkv=4, d=64, steps=40, r_d=0.5, recompress_every=1, cfg_id=22)
+    assert lockstep(ctx, cfg, 33, [(0, 0), (0, 1)]) <= 2
+    cfg = wl.DecodeConfig("dec_keepall", B=1, L=1, H=16, Hkv=2, d=128, steps=20, r_d=1.0, recompress_every=4, cfg_id=23)
+    assert lockstep(ctx, cfg, 300, [(0, 0)]) == 0
+
+
+def test_decode_empty_prefill_region(ctx):
+    cfg = wl.DecodeConfig("dec_m0", B=1, L=1, H=4, Hkv=2, d=128, steps=12, r_d=0.5, recompress_every=4, cfg_id=24)
+    counts = np.zeros((1, 1), np.int32)
+    assert lockstep(ctx, cfg, 8, [(0, 0)], counts) <= 1
+
+
+def test_decode_exact_ties_go_to_lower_index(ctx):
+    """All-zero queries: every entry's step weight is identical, so survivors are decided by age and,
+    among equals, by index -- same rule as the oracle pins."""
+    cfg = wl.DecodeConfig("dec_ties", B=1, L=1, H=4, Hkv=2, d=128, steps=8, r_d=0.5, recompress_every=4, cfg_id=25)
+    Kc, kept = wl.random_prefill_cache(cfg, 16, "cuda")
+    gpu = GpuDecoder(ctx, cfg, Kc, kept)
+    z = lambda *s: torch.zeros(*s, dtype=torch.bfloat16, device="cuda")
+    for _ in range(4):
+        gpu.step(z(1, 1, 4, 128), z(1, 1, 2, 128), z(1, 1, 2, 128))
+    torch.cuda.synchronize()
+    assert gpu.state.n_dec == 2 and gpu.born[0, 0, :2].tolist() == [0, 1]
+
+
+def test_decode_full_region_is_an_error(ctx):
+    cfg = wl.DecodeConfig("dec_full", B=1, L=1, H=4, Hkv=2, d=128, steps=4, r_d=1.0, recompress_every=1, cfg_id=26)
+    Kc, kept = wl.random_prefill_cache(cfg, 8, "cuda")
+    gpu = GpuDecoder(ctx, cfg, Kc, kept, Dcap=2)
+    q, k, v = wl.decode_step_inputs(cfg, 0, "cuda")
+    gpu.step(q, k, v); gpu.step(q, k, v)
+    with pytest.raises(skv.ShotKVError):
+        gpu.step(q, k, v)
+
+
+def test_decode_config4_shape_sampled_units(ctx):
+    """Config 4's shape (batch 8 x 32 layers, 3276 kept prefill keys, evict every 32 steps) for
+    three eviction cycles; the oracle follows three sampled (sequence, layer) units."""
+    cfg = wl.DECODE_CONFIG
+    ties = lockstep(ctx, cfg, 3276, [(0, 0), (3, 17), (7, 31)], steps=96)
+    assert ties <= 3

