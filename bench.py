@@ -1,0 +1,434 @@
+#!/usr/bin/env python
+"""Benchmark of the ShotKV hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One "step" is one pass of the prefill hot path (window scoring, per-shot reduce, shot selection,
+K/V compaction) over one batch of the long-context workload (config 3: 4 prompts x 32 layers x
+32,768 tokens, 8 KV heads, d=128, window 64, budget 10%).  `value` is prompt tokens compressed
+per second with the inputs resident in HBM; `e2e` is the same through the host-buffer entry
+point with the host<->device copies inside the timed region; `decode` reports decode steps/s on
+config 4 (batch 8 x 32 layers, 1,024 steps, evict to 25% every 32 steps) starting from a
+config-2-shaped compressed cache.  Rank 0 prints one JSON line.
+
+Multi-GPU: (prompt, layer) units are independent, so each rank compresses its own batch of
+prompts (weak scaling); the only communication is the barrier and the max-over-ranks of the
+device-side time.
+
+`--impl reference` times the fp64 CPU oracle on the host cores on a bounded sample of the same
+workload and prints the same line shape.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2502_01941_b200 import workloads as wl
+
+METRIC = "prompt tokens compressed/sec"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+
+
+# ------------------------------------------------------------------ small utilities
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a timed region runs."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-i", str(self.idx), "-lms", "50"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self, t_begin: float | None = None, t_end: float | None = None) -> dict:
+        """Ends sampling; keeps the samples whose timestamp lies in [t_begin, t_end] (wall clock)."""
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.06)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        import datetime
+        sm, mx, reasons = [], [], set()
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                if t_begin is not None and not (t_begin - 0.05 <= ts <= t_end + 0.05):
+                    continue
+                sm.append(float(parts[1])); mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_setup(n_gpus: int):
+    """(rank, world, local_rank); initialises NCCL only when launched under torchrun with N > 1."""
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=torch.device("cuda", local))
+    return rank, world, local
+
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    if world == 1:
+        return ms
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------ workloads
+def rank_config(cfg: wl.PrefillConfig, rank: int) -> wl.PrefillConfig:
+    return cfg if rank == 0 else cfg.replace(cfg_id=cfg.cfg_id + 1000 * rank)
+
+
+def algorithmic_bytes(cfg, kept_count: np.ndarray) -> dict:
+    """Bytes the method itself must move per step: all of K read once, and the kept K and V rows
+    read and written once each (actual kept counts)."""
+    row = cfg.d * 2
+    k_read = cfg.B * cfg.L * cfg.Hkv * cfg.N * row
+    gathered = int(kept_count.sum()) * cfg.Hkv * row * 2 * 2          # K and V, read + write
+    return {"k_read": k_read, "kv_gathered": gathered, "total": k_read + gathered}
+
+
+# ------------------------------------------------------------------ our arm
+def run_ours(args):
+    import paper_2502_01941_b200 as skv
+    from paper_2502_01941_b200.build import build_library
+    build_library()
+    rank, world, local = dist_setup(args.gpus)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    ctx = skv.Context(local)
+    peak, peak_src = measured_peaks()
+
+    cfg = rank_config(wl.CONFIGS[args.workload], rank)
+    if args.batch or args.layers:       # reduced copies of the workload, for profiler captures only
+        cfg = cfg.replace(B=args.batch or cfg.B, L=args.layers or cfg.L,
+                          name=f"{cfg.name}[B={args.batch or cfg.B},L={args.layers or cfg.L}]")
+    dims = skv.make_dims(cfg.B, cfg.L, cfg.H, cfg.Hkv, cfg.d, cfg.N, cfg.W, cfg.S)
+    pol = skv.make_policy(r_p=cfg.r_p)
+    Q, K, V, off = wl.prefill_batch(cfg, dev)
+    Mcap = skv.shotkv_kept_capacity(dims, pol, off)
+    out = skv.alloc_prefill_outputs(dims, Mcap, device=dev)
+
+    def step():
+        skv.shotkv_prefill_compress(ctx, dims, pol, Q, K, V, off, out["shot_scores"], out["keep"], out["kept_idx"],
+                                    out["kept_count"], Mcap, out["Kc"], out["Vc"], None, 0, out["ws"])
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier(world)
+    skv.shotkv_profile_enable(ctx, True)
+    launches0 = skv.shotkv_launch_count(ctx)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(world)
+    t_begin = time.time()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier(world)
+    t_end = time.time()
+    clocks = sampler.stop(t_begin, t_end)
+    launches = skv.shotkv_launch_count(ctx) - launches0
+    ms_total = max_over_ranks(e0.elapsed_time(e1), world, dev)
+    ms_step = ms_total / args.steps
+    stages = np.array([skv.shotkv_profile_read(ctx, i) for i in range(min(args.steps, 64))])   # [calls][3]
+    skv.shotkv_profile_enable(ctx, False)
+    kept = out["kept_count"].cpu().numpy()
+    ab = algorithmic_bytes(cfg, kept)
+    score_ms, select_ms, compact_ms = [float(x) for x in stages.mean(axis=0)]
+    tokens = cfg.B * cfg.N * world
+    value = tokens / (ms_step * 1e-3)
+    achieved = ab["k_read"] / (score_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "window scoring (QK^T + softmax partials), one launch per step",
+                "achieved": round(achieved, 1), "peak": peak, "peak_source": peak_src, "unit": "GB/s",
+                "frac": round(achieved / peak, 4), "traffic": None,
+                "algorithmic_bytes_per_launch": ab["k_read"], "ms_per_launch": round(score_ms, 4)}
+    path = {"bytes_per_step": ab["total"], "k_read_bytes": ab["k_read"], "kv_gathered_bytes": ab["kv_gathered"],
+            "achieved_gbs": round(ab["total"] / (ms_step * 1e-3) / 1e9, 1),
+            "frac_of_measured_hbm": round(ab["total"] / (ms_step * 1e-3) / 1e9 / peak, 4),
+            "frac_of_nominal_8tbs": round(ab["total"] / (ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS, 4),
+            "stage_ms": {"score": round(score_ms, 4), "select": round(select_ms, 4), "compact": round(compact_ms, 4)},
+            "compact_gbs": round(ab["kv_gathered"] / (compact_ms * 1e-3) / 1e9, 1),
+            "kept_tokens_mean": float(kept.mean()), "budget_tokens": skv.shotkv_budget_tokens(dims, pol)}
+
+    result = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 in, f32 accumulate", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "L": cfg.L, "H": cfg.H, "Hkv": cfg.Hkv, "d": cfg.d, "N": cfg.N,
+                   "W": cfg.W, "S": cfg.S, "r_p": cfg.r_p, "l2": "inputs (K alone %.1f GB) larger than the 126 MB L2; no flush" % (ab["k_read"] / 1e9),
+                   "parallelism": f"{world} independent replica(s), one batch of prompts each"},
+        "roofline": roofline, "path": path, "clocks": clocks, "gpu_launches": int(launches),
+    }
+
+    # ---------------- end to end from host buffers (rank-local, same workload)
+    if not args.no_e2e:
+        result["e2e"] = e2e_leg(skv, ctx, cfg, dims, pol, Q, K, V, off, Mcap, world, dev, args)
+    # ---------------- decode leg
+    del Q, K, V, out
+    torch.cuda.empty_cache()
+    if not args.no_decode:
+        result["decode"] = decode_leg(skv, ctx, rank, world, dev, peak, args)
+    # ---------------- CPU baseline (rank 0, N = 1 only)
+    if rank == 0 and world == 1 and not args.no_cpu:
+        result["cpu_baseline"] = cpu_baseline(cfg, off, budget_s=args.cpu_seconds)
+    ctx.close()
+    if rank == 0:
+        print(json.dumps(result))
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def e2e_leg(skv, ctx, cfg, dims, pol, Q, K, V, off, Mcap, world, dev, args) -> dict:
+    """Same metric through shotkv_prefill_compress_host: pinned host inputs and outputs, the
+    host->device copies of Q/K/V and the device->host copies of every result inside the timing."""
+    try:
+        hQ = torch.empty(Q.shape, dtype=Q.dtype, pin_memory=True); hQ.copy_(Q)
+        hK = torch.empty(K.shape, dtype=K.dtype, pin_memory=True); hK.copy_(K)
+        hV = torch.empty(V.shape, dtype=V.dtype, pin_memory=True); hV.copy_(V)
+        ho = skv.alloc_prefill_outputs(dims, Mcap, device="cpu")
+        for k in ("shot_scores", "keep", "kept_idx", "kept_count", "Kc", "Vc"):
+            ho[k] = ho[k].pin_memory()
+        arena = torch.empty(skv.shotkv_host_arena_bytes(dims, Mcap), dtype=torch.uint8, device=dev)
+    except RuntimeError as e:
+        return {"value": None, "unit": UNIT, "error": f"could not allocate pinned host buffers: {str(e)[:100]}"}
+    h2d = sum(t.numel() * t.element_size() for t in (hQ, hK, hV))
+    d2h = sum(ho[k].numel() * ho[k].element_size() for k in ("shot_scores", "keep", "kept_idx", "kept_count", "Kc", "Vc"))
+
+    def step():
+        skv.shotkv_prefill_compress_host(ctx, dims, pol, hQ, hK, hV, off, ho["shot_scores"], ho["keep"], ho["kept_idx"],
+                                         ho["kept_count"], Mcap, ho["Kc"], ho["Vc"], arena)
+    steps = max(2, min(args.steps, args.e2e_steps))
+    step()
+    barrier(world)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    barrier(world)
+    ms = max_over_ranks(e0.elapsed_time(e1), world, dev) / steps
+    return {"value": round(cfg.B * cfg.N * world / (ms * 1e-3), 1), "unit": UNIT, "ms_per_step": round(ms, 3),
+            "steps": steps, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+            "api": "shotkv_prefill_compress_host"}
+
+
+def decode_leg(skv, ctx, rank, world, dev, peak, args) -> dict:
+    """Config 4: batch 8 x 32 layers; the compressed prefill cache comes from running Phase 1 on a
+    config-2-shaped batch of 8 prompts; then 1,024 decode steps, evicting to 25% every 32 steps."""
+    dc = wl.DECODE_CONFIG
+    if args.decode_steps:
+        import dataclasses
+        dc = dataclasses.replace(dc, steps=args.decode_steps)
+    pc = rank_config(wl.CONFIGS[2].replace(B=dc.B), rank)
+    dims = skv.make_dims(pc.B, pc.L, pc.H, pc.Hkv, pc.d, pc.N, pc.W, pc.S)
+    pol = skv.make_policy(r_p=pc.r_p, r_d=dc.r_d, recompress_every=dc.recompress_every)
+    Q, K, V, off = wl.prefill_batch(pc, dev)
+    Mcap = skv.shotkv_kept_capacity(dims, pol, off)
+    out = skv.alloc_prefill_outputs(dims, Mcap, device=dev)
+    skv.shotkv_prefill_compress(ctx, dims, pol, Q, K, V, off, out["shot_scores"], out["keep"], out["kept_idx"],
+                                out["kept_count"], Mcap, out["Kc"], out["Vc"], None, 0, out["ws"])
+    torch.cuda.synchronize()
+    del Q, K, V
+    torch.cuda.empty_cache()
+    kept = out["kept_count"].cpu().numpy()
+    Dcap = skv.shotkv_decode_capacity(pol, dc.steps)
+    Kd = torch.zeros(dc.B, dc.L, dc.Hkv, Dcap, dc.d, dtype=torch.bfloat16, device=dev)
+    Vd = torch.zeros_like(Kd)
+    acc = torch.zeros(dc.B, dc.L, Dcap, device=dev)
+    born = torch.zeros(dc.B, dc.L, Dcap, dtype=torch.int32, device=dev)
+    ws = torch.empty(skv.shotkv_decode_workspace_bytes(dims, Dcap), dtype=torch.uint8, device=dev)
+    # the step inputs are drawn before the timed region: one (q, k, v) triple per step
+    n_in = 64
+    ins = [wl.decode_step_inputs(dc, s, dev) for s in range(n_in)]
+
+    def run(steps, profile=False):
+        st = skv.shotkv_decode_init(ctx, dims, pol, Dcap, Mcap, Kd, Vd, acc, born, ws)
+        bytes_read = 0
+        for s in range(steps):
+            q, k, v = ins[s % n_in]
+            bytes_read += (int(kept.sum()) + (st.n_dec + 1) * dc.B * dc.L) * dc.Hkv * dc.d * 2
+            skv.shotkv_decode_step(ctx, st, q, k, v, out["Kc"], out["kept_count"])
+        return bytes_read
+
+    run(max(args.warmup, 3) * 8)
+    barrier(world)
+    skv.shotkv_profile_enable(ctx, True)
+    l0 = skv.shotkv_launch_count(ctx)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    bytes_read = run(dc.steps)
+    e1.record()
+    barrier(world)
+    ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
+    launches = skv.shotkv_launch_count(ctx) - l0
+    st_ms = np.array([skv.shotkv_profile_read(ctx, i)[:2] for i in range(64)])
+    skv.shotkv_profile_enable(ctx, False)
+    per_step_bytes = bytes_read / dc.steps
+    score_ms = float(st_ms[:, 0].mean())
+    return {"metric": "decode steps/sec", "value": round(dc.steps * world / (ms * 1e-3), 1), "unit": "steps/s",
+            "note": "one step = all 8 sequences x 32 layers of one replica; value sums the replicas",
+            "steps": dc.steps, "ms_per_step": round(ms / dc.steps, 4), "gpu_launches": int(launches),
+            "config": {"workload": dc.name, "B": dc.B, "L": dc.L, "H": dc.H, "Hkv": dc.Hkv, "d": dc.d,
+                       "prefill_kept_mean": float(kept.mean()), "r_d": dc.r_d, "recompress_every": dc.recompress_every,
+                       "Dcap": Dcap},
+            "roofline": {"bound": "hbm", "kernel": "decode score kernel (last 64 steps)",
+                         "achieved": round(per_step_bytes / (score_ms * 1e-3) / 1e9, 1), "peak": peak, "unit": "GB/s",
+                         "frac": round(per_step_bytes / (score_ms * 1e-3) / 1e9 / peak, 4), "traffic": None,
+                         "algorithmic_bytes_per_launch": int(per_step_bytes), "ms_per_launch": round(score_ms, 4)},
+            "path_frac_of_measured_hbm": round(per_step_bytes / (ms / dc.steps * 1e-3) / 1e9 / peak, 4)}
+
+
+# ------------------------------------------------------------------ the oracle, timed
+def oracle_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return 1
+
+
+def oracle_unit_seconds(cfg, b, l, off_b) -> float:
+    """Times the oracle, as it stands, on one (prompt, layer) unit of the workload."""
+    from oracle import shotkv_oracle as O
+    Q, K, V = wl.prefill_unit(cfg, b, l, off_b, "cpu")
+    q, k, v = wl.bf16_to_f64(Q), wl.bf16_to_f64(K), wl.bf16_bits(V)
+    t0 = time.perf_counter()
+    O.prefill_compress(q, k, v, off_b, cfg.r_p)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(cfg, off, budget_s: float = 20.0) -> dict:
+    """The fp64 oracle on the host cores, on as many (prompt 0, layer l) units of the same workload
+    as fit in about `budget_s` seconds.  One unit = N tokens of one layer; a prompt is L units."""
+    t_total, n_units = 0.0, 0
+    while t_total < budget_s and n_units < cfg.L:
+        t_total += oracle_unit_seconds(cfg, 0, n_units, off[0])
+        n_units += 1
+    tokens_per_s = cfg.N / (t_total / n_units * cfg.L)
+    return {"value": round(tokens_per_s, 2), "unit": UNIT, "cores": oracle_threads(), "host_cpus": os.cpu_count(),
+            "kind": "oracle", "sample": f"{n_units} of {cfg.B * cfg.L} (prompt, layer) units of {cfg.name} "
+                                        f"({n_units * cfg.N} token-layers) in {t_total:.1f} s; scaled to whole prompts"}
+
+
+def run_reference(args):
+    """The reference arm is the oracle itself (there is no reference implementation to install):
+    each step compresses a bounded sample -- one (prompt, layer) unit -- of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = wl.CONFIGS[args.workload]
+    off = wl.all_shot_offsets(cfg)
+    steps, warm = min(args.steps, 8), min(max(args.warmup, 1), 2)
+    for i in range(warm):
+        oracle_unit_seconds(cfg, 0, i % cfg.L, off[0])
+    t = [oracle_unit_seconds(cfg, 0, (warm + i) % cfg.L, off[0]) for i in range(steps)]
+    sec = sum(t) / steps
+    value = cfg.N / (sec * cfg.L)
+    line = {"impl": "reference", "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": warm, "ms_per_step": round(sec * 1e3, 2), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "B": cfg.B, "L": cfg.L, "H": cfg.H, "Hkv": cfg.Hkv, "d": cfg.d, "N": cfg.N,
+                       "W": cfg.W, "S": cfg.S, "r_p": cfg.r_p},
+            "cpu_baseline": {"value": round(value, 2), "unit": UNIT, "kind": "oracle", "cores": oracle_threads(),
+                             "sample": f"each step = one (prompt, layer) unit of {cfg.name} ({cfg.N} token-layers); "
+                                       f"tokens/s scaled by L = {cfg.L} layers per prompt"},
+            "e2e": {"value": round(value, 2), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3], help="prefill config timed as the step")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-seconds", type=float, default=20.0)
+    ap.add_argument("--batch", type=int, default=0, help="override B (profiler captures of a smaller case)")
+    ap.add_argument("--layers", type=int, default=0, help="override L (profiler captures of a smaller case)")
+    ap.add_argument("--decode-steps", type=int, default=0, help="override the number of decode steps")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

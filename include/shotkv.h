@@ -210,6 +210,18 @@ SHOTKV_API int shotkv_decode_step(shotkv_ctx* ctx, shotkv_decode_state* state,
                        const shotkv_bf16* q, const shotkv_bf16* k_new, const shotkv_bf16* v_new,
                        const shotkv_bf16* Kc, const int32_t* kept_count, void* stream);
 
+/* ---- instrumentation (used by the benchmark; not part of the method) ------------------------ */
+
+/* When enabled, shotkv_prefill_compress (single-pass form) and shotkv_decode_step record CUDA
+ * events on their stream at their stage boundaries; the last 64 calls are retained.  */
+SHOTKV_API int shotkv_profile_enable(shotkv_ctx* ctx, int enable);
+/* Stage durations in milliseconds of the profiled call made `calls_back` calls ago (0 = latest);
+ * waits for that call to finish.  Prefill: {score+per-shot reduce, select, compact};
+ * decode: {score kernel, accumulate+evict, -1}.  Returns the number of stages or a negative error. */
+SHOTKV_API int shotkv_profile_read(shotkv_ctx* ctx, int calls_back, float* stage_ms /* [3] */);
+/* Kernels launched through this context since it was created. */
+SHOTKV_API uint64_t shotkv_launch_count(const shotkv_ctx* ctx);
+
 #ifdef __cplusplus
 }
 #endif

@@ -32,6 +32,7 @@ EXPORTS = [
     "shotkv_prefill_score", "shotkv_select_shots", "shotkv_compact_kv", "shotkv_prefill_compress",
     "shotkv_host_arena_bytes", "shotkv_prefill_compress_host",
     "shotkv_decode_workspace_bytes", "shotkv_decode_capacity", "shotkv_decode_init", "shotkv_decode_step",
+    "shotkv_profile_enable", "shotkv_profile_read", "shotkv_launch_count",
 ]
 
 
@@ -90,6 +91,9 @@ def lib() -> C.CDLL:
         "shotkv_decode_capacity": (i32, [PP, i32]),
         "shotkv_decode_init": (C.c_int, [vp, PD, PP, i32, i32, vp, vp, vp, vp, vp, sz, C.POINTER(DecodeState)]),
         "shotkv_decode_step": (C.c_int, [vp, C.POINTER(DecodeState), vp, vp, vp, vp, vp, vp]),
+        "shotkv_profile_enable": (C.c_int, [vp, C.c_int]),
+        "shotkv_profile_read": (C.c_int, [vp, C.c_int, C.POINTER(C.c_float)]),
+        "shotkv_launch_count": (C.c_uint64, [vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(L, name)
@@ -290,6 +294,20 @@ def shotkv_decode_step(ctx: Context, state: DecodeState, q, k_new, v_new, Kc, ke
                                   _ptr(Kc, device="cuda", dtype=torch.bfloat16, name="Kc"),
                                   _ptr(kept_count, device="cuda", dtype=torch.int32, name="kept_count"), _stream(stream))
     return ctx.check(rc)
+
+
+def shotkv_profile_enable(ctx: Context, enable: bool) -> int:
+    return ctx.check(lib().shotkv_profile_enable(ctx._h, int(bool(enable))))
+
+
+def shotkv_profile_read(ctx: Context, calls_back: int = 0) -> list:
+    ms = (C.c_float * 3)()
+    n = ctx.check(lib().shotkv_profile_read(ctx._h, int(calls_back), ms))
+    return [float(ms[i]) for i in range(n)]
+
+
+def shotkv_launch_count(ctx: Context) -> int:
+    return int(lib().shotkv_launch_count(ctx._h))
 
 
 def alloc_prefill_outputs(dims: Dims, Mcap: int, device="cuda", token_importance: bool = False) -> dict:

@@ -24,6 +24,7 @@ constexpr int kPieceMaxKeys = 512;     // longest key range one scoring work ite
 constexpr int kMaxShots = 8192;
 constexpr int kStageSlots = 4;
 constexpr size_t kStageSlotBytes = 1u << 20;
+constexpr int kProfSlots = 64;
 
 inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
@@ -36,6 +37,12 @@ struct shotkv_ctx {
     unsigned char* stage = nullptr;
     cudaEvent_t stage_done[kStageSlots] = {};
     int stage_next = 0;
+    // optional stage timing: a ring of event sets, one per profiled call
+    bool prof = false;
+    cudaEvent_t prof_ev[kProfSlots][4] = {};
+    int prof_marks[kProfSlots] = {};
+    int prof_calls = 0;
+    unsigned long long launches = 0;   // kernels launched through this context
 };
 
 namespace {
@@ -56,6 +63,26 @@ int fail(shotkv_ctx* ctx, int code, const char* fmt, ...) {
         if (e__ != cudaSuccess)                                                                 \
             return fail(ctx, SHOTKV_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e__)); \
     } while (0)
+
+// After every kernel launch: count it and surface launch errors.
+#define LAUNCH_CHECK(ctx)                    \
+    do {                                     \
+        (ctx)->launches += 1;                \
+        CUDA_TRY(ctx, cudaGetLastError());   \
+    } while (0)
+
+// Records the next stage boundary of the current profiled call (no-op unless profiling is on).
+void prof_begin(shotkv_ctx* ctx) {
+    if (!ctx->prof) return;
+    ctx->prof_calls += 1;
+    ctx->prof_marks[(ctx->prof_calls - 1) % kProfSlots] = 0;
+}
+void prof_mark(shotkv_ctx* ctx, cudaStream_t stream) {
+    if (!ctx->prof || ctx->prof_calls == 0) return;
+    const int slot = (ctx->prof_calls - 1) % kProfSlots;
+    int& m = ctx->prof_marks[slot];
+    if (m < 4) cudaEventRecord(ctx->prof_ev[slot][m++], stream);
+}
 
 int check_dims(const shotkv_dims* d, const char** why) {
     if (!d) { *why = "dims is NULL"; return SHOTKV_ERR_INVALID_ARG; }
@@ -200,7 +227,7 @@ int launch_score_t(shotkv_ctx* ctx, const ScoreParams& sp, int U, cudaStream_t s
     }
     dim3 grid((sp.P + sp.ppc - 1) / sp.ppc, U);
     score_mma_kernel<D, MB, COLSUM><<<grid, 256, smem, stream>>>(sp);
-    CUDA_TRY(ctx, cudaGetLastError());
+    LAUNCH_CHECK(ctx);
     return SHOTKV_OK;
 }
 
@@ -257,11 +284,12 @@ int run_stats(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const
     if (rc) return rc;
     const int U = d->B * d->L * d->Hkv;
     ScoreParams sp = base_params(d, Q, K, w, P);
+    prof_mark(ctx, stream);
     rc = launch_score<false>(ctx, d, sp, U, stream);
     if (rc) return rc;
     if (need_rows) {
         row_stats_kernel<<<U, 256, 0, stream>>>(w.part_m, w.part_z, P, sp.R, sp.Rpad, w.row_m, w.row_invz);
-        CUDA_TRY(ctx, cudaGetLastError());
+        LAUNCH_CHECK(ctx);
     }
     *P_out = P;
     return SHOTKV_OK;
@@ -277,7 +305,7 @@ int run_select(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_policy* p, co
     }
     select_shots_kernel<<<d->B * d->L, kSelectThreads, smem, stream>>>(shot_scores, w.off, d->L, d->N, d->S, budget_of(d, p),
                                                                      p->select_mode, Mcap, keep, kept_idx, kept_count);
-    CUDA_TRY(ctx, cudaGetLastError());
+    LAUNCH_CHECK(ctx);
     return SHOTKV_OK;
 }
 
@@ -292,7 +320,7 @@ int run_compact(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* K, con
         compact_kv_kernel<128><<<grid, 256, 0, stream>>>((const uint4*)K, (const uint4*)V, kept_idx, kept_count, d->Hkv, d->N, Mcap, (uint4*)Kc, (uint4*)Vc);
     else
         compact_kv_kernel<64><<<grid, 256, 0, stream>>>((const uint4*)K, (const uint4*)V, kept_idx, kept_count, d->Hkv, d->N, Mcap, (uint4*)Kc, (uint4*)Vc);
-    CUDA_TRY(ctx, cudaGetLastError());
+    LAUNCH_CHECK(ctx);
     return SHOTKV_OK;
 }
 
@@ -338,6 +366,9 @@ void shotkv_destroy(shotkv_ctx* ctx) {
             cudaEventDestroy(ctx->stage_done[i]);
         }
     if (ctx->stage) cudaFreeHost(ctx->stage);
+    for (int i = 0; i < kProfSlots; ++i)
+        for (int j = 0; j < 4; ++j)
+            if (ctx->prof_ev[i][j]) cudaEventDestroy(ctx->prof_ev[i][j]);
     delete ctx;
 }
 
@@ -418,7 +449,7 @@ int shotkv_select_shots(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_p
     if (token_importance && dims->S > 0) {
         dim3 grid(dims->S, dims->B * dims->L);
         shot_score_from_tokens_kernel<<<grid, 128, 0, stream>>>(token_importance, w.off, dims->L, dims->Hkv, dims->N, dims->S, shot_scores);
-        CUDA_TRY(ctx, cudaGetLastError());
+        LAUNCH_CHECK(ctx);
     }
     if ((rc = run_select(ctx, dims, policy, w, shot_scores, keep, kept_idx, kept_count, Mcap, stream))) return rc;
     if (orc > 0) fail(ctx, orc, "always-kept tokens (%d) exceed the budget (%d) for some prompt", worst, budget_of(dims, policy));
@@ -467,6 +498,7 @@ int shotkv_prefill_compress(shotkv_ctx* ctx, const shotkv_dims* dims, const shot
     const PrefillWs w = carve(dims, ws);
     if ((rc = upload_small(ctx, w.off, offsets_host, (size_t)dims->B * (dims->S + 1) * 4, stream))) return rc;
     int P = 0;
+    prof_begin(ctx);
     if ((rc = run_stats(ctx, dims, Qwin, K, w, offsets_host, false, &P, stream))) return rc;
     const int U = dims->B * dims->L * dims->Hkv;
     const int R = (dims->H / dims->Hkv) * dims->W, Rpad = rpad_of(dims);
@@ -475,12 +507,15 @@ int shotkv_prefill_compress(shotkv_ctx* ctx, const shotkv_dims* dims, const shot
             shot_mass_kernel<128><<<U, 128, 0, stream>>>(w.part_m, w.part_z, w.piece_seg, P, R, Rpad, dims->L, dims->Hkv, dims->S, w.unit_shot);
         else
             shot_mass_kernel<256><<<U, 256, 0, stream>>>(w.part_m, w.part_z, w.piece_seg, P, R, Rpad, dims->L, dims->Hkv, dims->S, w.unit_shot);
-        CUDA_TRY(ctx, cudaGetLastError());
+        LAUNCH_CHECK(ctx);
         shot_score_from_mass_kernel<<<dims->B * dims->L, 128, 0, stream>>>(w.unit_shot, w.off, dims->L, dims->Hkv, dims->S, shot_scores);
-        CUDA_TRY(ctx, cudaGetLastError());
+        LAUNCH_CHECK(ctx);
     }
+    prof_mark(ctx, stream);
     if ((rc = run_select(ctx, dims, policy, w, shot_scores, keep, kept_idx, kept_count, Mcap, stream))) return rc;
+    prof_mark(ctx, stream);
     if ((rc = run_compact(ctx, dims, K, V, kept_idx, kept_count, Mcap, Kc, Vc, stream))) return rc;
+    prof_mark(ctx, stream);
     if (orc > 0) fail(ctx, orc, "always-kept tokens (%d) exceed the budget (%d) for some prompt", worst, budget_of(dims, policy));
     return orc;
 }
@@ -624,6 +659,8 @@ int shotkv_decode_step(shotkv_ctx* ctx, shotkv_decode_state* st, const shotkv_bf
     p.H = d.H; p.Hkv = d.Hkv; p.G = d.H / d.Hkv; p.Mcap = st->Mcap; p.Dcap = st->Dcap; p.n_old = st->n_dec;
     p.scale_log2 = kLog2e / sqrtf((float)d.d);
     const size_t smem = (size_t)8 * st->Dcap * 4 + (8 * 8 * 2 + 16) * 4;
+    prof_begin(ctx);
+    prof_mark(ctx, stream);
     if (d.d == 128) {
         CUDA_TRY(ctx, cudaFuncSetAttribute(decode_score_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
         decode_score_kernel<128><<<U, 256, smem, stream>>>(p);
@@ -631,9 +668,10 @@ int shotkv_decode_step(shotkv_ctx* ctx, shotkv_decode_state* st, const shotkv_bf
         CUDA_TRY(ctx, cudaFuncSetAttribute(decode_score_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
         decode_score_kernel<64><<<U, 256, smem, stream>>>(p);
     }
-    CUDA_TRY(ctx, cudaGetLastError());
+    LAUNCH_CHECK(ctx);
+    prof_mark(ctx, stream);
     decode_accumulate_kernel<<<BL, 128, 0, stream>>>(partial, d.Hkv, st->Dcap, st->n_dec, st->T, st->acc, st->born);
-    CUDA_TRY(ctx, cudaGetLastError());
+    LAUNCH_CHECK(ctx);
     st->n_dec += 1;
     st->T += 1;
     if (st->T % st->policy.recompress_every == 0) {
@@ -644,19 +682,49 @@ int shotkv_decode_step(shotkv_ctx* ctx, shotkv_decode_state* st, const shotkv_bf
             const size_t rs = (size_t)n * 16 + (kSelectThreads + 1) * 4 + 16;
             CUDA_TRY(ctx, cudaFuncSetAttribute(decode_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
             decode_rank_kernel<<<BL, kSelectThreads, rs, stream>>>(st->acc, st->born, st->Dcap, n, k, keep_pos);
-            CUDA_TRY(ctx, cudaGetLastError());
+            LAUNCH_CHECK(ctx);
             if (k > 0) {
                 dim3 grid(U, 2);
                 if (d.d == 128)
                     decode_compact_kernel<128><<<grid, 256, 0, stream>>>((__nv_bfloat16*)st->Kd, (__nv_bfloat16*)st->Vd, keep_pos, d.Hkv, st->Dcap, k);
                 else
                     decode_compact_kernel<64><<<grid, 256, 0, stream>>>((__nv_bfloat16*)st->Kd, (__nv_bfloat16*)st->Vd, keep_pos, d.Hkv, st->Dcap, k);
-                CUDA_TRY(ctx, cudaGetLastError());
+                LAUNCH_CHECK(ctx);
             }
             st->n_dec = k;
         }
     }
+    prof_mark(ctx, stream);
     return SHOTKV_OK;
 }
+
+// ---- instrumentation ------------------------------------------------------------------------
+int shotkv_profile_enable(shotkv_ctx* ctx, int enable) {
+    int rc = set_device(ctx);
+    if (rc) return rc;
+    if (enable && !ctx->prof_ev[0][0]) {
+        for (int i = 0; i < kProfSlots; ++i)
+            for (int j = 0; j < 4; ++j) CUDA_TRY(ctx, cudaEventCreate(&ctx->prof_ev[i][j]));
+    }
+    ctx->prof = enable != 0;
+    ctx->prof_calls = 0;
+    return SHOTKV_OK;
+}
+
+int shotkv_profile_read(shotkv_ctx* ctx, int calls_back, float* stage_ms) {
+    int rc = set_device(ctx);
+    if (rc) return rc;
+    if (!stage_ms || calls_back < 0 || calls_back >= kProfSlots || calls_back >= ctx->prof_calls)
+        return fail(ctx, SHOTKV_ERR_INVALID_ARG, "no profiled call %d calls back", calls_back);
+    const int slot = (ctx->prof_calls - 1 - calls_back) % kProfSlots;
+    const int m = ctx->prof_marks[slot];
+    for (int i = 0; i < 3; ++i) stage_ms[i] = -1.f;
+    if (m < 2) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "that call recorded no stages");
+    CUDA_TRY(ctx, cudaEventSynchronize(ctx->prof_ev[slot][m - 1]));
+    for (int i = 0; i + 1 < m; ++i) CUDA_TRY(ctx, cudaEventElapsedTime(&stage_ms[i], ctx->prof_ev[slot][i], ctx->prof_ev[slot][i + 1]));
+    return m - 1;
+}
+
+uint64_t shotkv_launch_count(const shotkv_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 }  // extern "C"
