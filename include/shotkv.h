@@ -131,6 +131,28 @@ SHOTKV_API int shotkv_select_shots(shotkv_ctx* ctx, const shotkv_dims* dims, con
                         float* shot_scores, uint8_t* keep, int32_t* kept_idx, int32_t* kept_count,
                         int32_t Mcap, void* ws, size_t ws_bytes, void* stream);
 
+/* shotkv_select_shots for callers that cannot allocate device memory (the paper has no
+ * counterpart; this is a packaging variant, the arithmetic is that of shotkv_select_shots).
+ * Some hosts of this library may not call cudaMalloc at the point where they compress a prompt:
+ * an inference server that handed all of HBM to its own pool at start-up, a plug-in running
+ * inside another runtime's stream callback or memory-frozen region, a real-time loop that bans
+ * allocator calls.  shotkv_select_shots needs a caller-supplied workspace only to hold the device
+ * copy of the shot boundaries; here that copy lives in a fixed table inside the library image
+ * (SHOTKV_STATIC_OFFSETS_MAX = 65536 int32 entries, 256 KB, resident on every GPU that loads the
+ * library until the process exits).  The call performs no cudaMalloc/cudaFree and uses no
+ * allocating library routine.
+ *   - Limit: B*(S+1) <= 65536, else SHOTKV_ERR_UNSUPPORTED_SHAPE (use the workspace form).
+ *   - The first call on each device looks up the table's device address; make that first call
+ *     outside any stream capture.
+ *   - All calls on a device share the one table, and it keeps the previous call's contents: each
+ *     call overwrites every entry it reads, but two calls that overlap on the GPU (different
+ *     streams, or the same stream from two threads) race on it.  Serialise them.
+ * All other arguments, outputs and return codes are those of shotkv_select_shots.  */
+SHOTKV_API int shotkv_select_shots_static(shotkv_ctx* ctx, const shotkv_dims* dims,
+                               const shotkv_policy* policy, const float* token_importance,
+                               const int32_t* offsets_host, float* shot_scores, uint8_t* keep,
+                               int32_t* kept_idx, int32_t* kept_count, int32_t Mcap, void* stream);
+
 /* Compress (Section 5.1, Compress equation): gathers the kept rows of every KV head of a layer.
  *   Kc[b][l][g][j] = K[b][l][g][kept_idx[b][l][j]]  for j < kept_count[b][l]; same for V.
  *   K, V   device [B][L][Hkv][N][d] bf16     Kc, Vc  device [B][L][Hkv][Mcap][d] bf16

@@ -32,7 +32,7 @@ EXPORTS = [
     "shotkv_prefill_score", "shotkv_select_shots", "shotkv_compact_kv", "shotkv_prefill_compress",
     "shotkv_host_arena_bytes", "shotkv_prefill_compress_host",
     "shotkv_decode_workspace_bytes", "shotkv_decode_capacity", "shotkv_decode_init", "shotkv_decode_step",
-    "shotkv_profile_enable", "shotkv_profile_read", "shotkv_launch_count",
+    "shotkv_profile_enable", "shotkv_profile_read", "shotkv_launch_count", "shotkv_select_shots_static",
 ]
 
 
@@ -83,6 +83,7 @@ def lib() -> C.CDLL:
         "shotkv_workspace_bytes": (sz, [PD]),
         "shotkv_prefill_score": (C.c_int, [vp, PD, vp, vp, vp, vp, sz, vp]),
         "shotkv_select_shots": (C.c_int, [vp, PD, PP, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp]),
+        "shotkv_select_shots_static": (C.c_int, [vp, PD, PP, vp, vp, vp, vp, vp, vp, i32, vp]),
         "shotkv_compact_kv": (C.c_int, [vp, PD, vp, vp, vp, vp, i32, vp, vp, vp]),
         "shotkv_prefill_compress": (C.c_int, [vp, PD, PP, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, u32, vp, sz, vp]),
         "shotkv_host_arena_bytes": (sz, [PD, i32]),
@@ -212,6 +213,23 @@ def shotkv_select_shots(ctx: Context, dims: Dims, policy: Policy, token_importan
                                    _ptr(kept_count, device="cuda", dtype=torch.int32, name="kept_count"),
                                    int(Mcap), _ptr(ws, device="cuda", name="ws"), ws.numel() * ws.element_size(),
                                    _stream(stream))
+    return ctx.check(rc)
+
+
+def shotkv_select_shots_static(ctx: Context, dims: Dims, policy: Policy, token_importance, offsets, shot_scores, keep,
+                               kept_idx, kept_count, Mcap: int, stream=None) -> int:
+    """shotkv_select_shots without a workspace argument: for hosts that may not allocate device
+    memory when they compress (the boundary table sits in a fixed 256 KB array inside the library;
+    B*(S+1) <= 65536).  Calls on one device must not overlap on the GPU."""
+    o = _offsets(offsets)
+    rc = lib().shotkv_select_shots_static(ctx._h, C.byref(dims), C.byref(policy),
+                                          _ptr(token_importance, device="cuda", dtype=torch.float32, name="token_importance"),
+                                          o.ctypes.data_as(C.c_void_p),
+                                          _ptr(shot_scores, device="cuda", dtype=torch.float32, name="shot_scores"),
+                                          _ptr(keep, device="cuda", dtype=torch.uint8, name="keep"),
+                                          _ptr(kept_idx, device="cuda", dtype=torch.int32, name="kept_idx"),
+                                          _ptr(kept_count, device="cuda", dtype=torch.int32, name="kept_count"),
+                                          int(Mcap), _stream(stream))
     return ctx.check(rc)
 
 

@@ -456,6 +456,64 @@ int shotkv_select_shots(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_p
     return orc;
 }
 
+// ---- selection without any caller- or library-allocated scratch ------------------------------
+// Device copy of the shot boundaries for shotkv_select_shots_static.  It lives in the library
+// image: every GPU that loads the library holds these 256 KB until the process exits.
+#define SHOTKV_STATIC_OFFSETS_MAX 65536
+static __device__ __align__(256) int32_t g_static_offsets[SHOTKV_STATIC_OFFSETS_MAX];
+
+namespace {
+// In host code `g_static_offsets` is only a handle; the address kernels can use has to be asked
+// for, per device, with that device current.
+int static_offsets_ptr(shotkv_ctx* ctx, int32_t** out) {
+    static int32_t* ptr_of_device[64] = {};
+    const int dev = ctx->device;
+    if (dev < 0 || dev >= 64) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "device index %d beyond 63", dev);
+    if (!ptr_of_device[dev]) {
+        int32_t* p = nullptr;
+        CUDA_TRY(ctx, cudaGetSymbolAddress((void**)&p, g_static_offsets));
+        if (!p) return fail(ctx, SHOTKV_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
+        ptr_of_device[dev] = p;
+    }
+    *out = ptr_of_device[dev];
+    return SHOTKV_OK;
+}
+}  // namespace
+
+int shotkv_select_shots_static(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_policy* policy,
+                               const float* token_importance, const int32_t* offsets_host, float* shot_scores,
+                               uint8_t* keep, int32_t* kept_idx, int32_t* kept_count, int32_t Mcap, void* stream_) {
+    int rc = set_device(ctx);
+    if (rc) return rc;
+    const char* why = "";
+    if ((rc = check_dims(dims, &why))) return fail(ctx, rc, "%s", why);
+    if ((rc = check_policy_prefill(policy, &why))) return fail(ctx, rc, "%s", why);
+    const long long entries = (long long)dims->B * (dims->S + 1);
+    if (entries > SHOTKV_STATIC_OFFSETS_MAX)
+        return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE,
+                    "B*(S+1) = %lld boundary entries exceed the built-in table of %d; use shotkv_select_shots with a workspace",
+                    entries, SHOTKV_STATIC_OFFSETS_MAX);
+    int worst = 0;
+    const int orc = check_offsets(dims, policy, offsets_host, &worst, &why);
+    if (orc < 0) return fail(ctx, orc, "%s", why);
+    if (!shot_scores || !keep || !kept_idx || !kept_count) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "output pointers must not be NULL");
+    const int need = budget_of(dims, policy) > worst ? budget_of(dims, policy) : worst;
+    if (Mcap < need) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "Mcap = %d but %d rows may be kept", Mcap, need);
+    cudaStream_t stream = (cudaStream_t)stream_;
+    PrefillWs w{};
+    if ((rc = static_offsets_ptr(ctx, &w.off))) return rc;
+    // every entry the kernels read is overwritten here, so nothing of an earlier call survives
+    if ((rc = upload_small(ctx, w.off, offsets_host, (size_t)entries * 4, stream))) return rc;
+    if (token_importance && dims->S > 0) {
+        dim3 grid(dims->S, dims->B * dims->L);
+        shot_score_from_tokens_kernel<<<grid, 128, 0, stream>>>(token_importance, w.off, dims->L, dims->Hkv, dims->N, dims->S, shot_scores);
+        LAUNCH_CHECK(ctx);
+    }
+    if ((rc = run_select(ctx, dims, policy, w, shot_scores, keep, kept_idx, kept_count, Mcap, stream))) return rc;
+    if (orc > 0) fail(ctx, orc, "always-kept tokens (%d) exceed the budget (%d) for some prompt", worst, budget_of(dims, policy));
+    return orc;
+}
+
 int shotkv_compact_kv(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_bf16* K, const shotkv_bf16* V,
                       const int32_t* kept_idx, const int32_t* kept_count, int32_t Mcap, shotkv_bf16* Kc, shotkv_bf16* Vc,
                       void* stream_) {
