@@ -175,7 +175,8 @@ __global__ void __launch_bounds__(kSelectThreads) decode_rank_kernel(float* __re
     int* tmp = ds + n;
     const int bl = blockIdx.x, tid = threadIdx.x;
     for (int j = tid; j < n; j += kSelectThreads) {
-        a[j] = acc[(size_t)bl * Dcap + j];
+        const float v = acc[(size_t)bl * Dcap + j];
+        a[j] = v == v ? v : SHOTKV_NEG_INF;      // keep the order total even if a score is NaN
         bs[j] = born[(size_t)bl * Dcap + j];
     }
     __syncthreads();

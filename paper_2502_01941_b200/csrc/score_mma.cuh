@@ -240,6 +240,11 @@ __global__ void row_stats_kernel(const float* __restrict__ part_m, const float* 
                                  int Rpad, float* __restrict__ row_m, float* __restrict__ row_invz) {
     const int u = blockIdx.x;
     for (int r = threadIdx.x; r < Rpad; r += blockDim.x) {
+        if (r >= R) {   // padding rows carry no weight; their partials may be anything
+            row_m[(size_t)u * Rpad + r] = 0.f;
+            row_invz[(size_t)u * Rpad + r] = 0.f;
+            continue;
+        }
         const float* pm = part_m + (size_t)u * P * Rpad + r;
         const float* pz = part_z + (size_t)u * P * Rpad + r;
         float m = SHOTKV_NEG_INF;

@@ -57,7 +57,10 @@ __global__ void __launch_bounds__(kSelectThreads) select_shots_kernel(
     const int always = pre + (N - qst);
     const int shot_budget = budget_tokens - always;
 
-    for (int i = tid; i < S; i += kSelectThreads) sc[i] = shot_scores[(size_t)bl * S + i];
+    for (int i = tid; i < S; i += kSelectThreads) {
+        const float v = shot_scores[(size_t)bl * S + i];
+        sc[i] = v == v ? v : SHOTKV_NEG_INF;     // a NaN score ranks last instead of breaking the total order
+    }
     __syncthreads();
     for (int i = tid; i < S; i += kSelectThreads) {
         const float v = sc[i];

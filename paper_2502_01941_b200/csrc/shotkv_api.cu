@@ -7,6 +7,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -14,6 +15,7 @@
 #include "common.cuh"
 #include "decode.cuh"
 #include "score_mma.cuh"
+#include "score_tc.cuh"
 #include "select_compact.cuh"
 
 using namespace shotkv;
@@ -43,6 +45,10 @@ struct shotkv_ctx {
     int prof_marks[kProfSlots] = {};
     int prof_calls = 0;
     unsigned long long launches = 0;   // kernels launched through this context
+    // error word that kernels with bounded waits raise; pinned host memory mapped into the device
+    int* err_host = nullptr;
+    int* err_dev = nullptr;
+    int sm_count = 148;
 };
 
 namespace {
@@ -259,7 +265,80 @@ ScoreParams base_params(const shotkv_dims* d, const shotkv_bf16* Q, const shotkv
 int set_device(shotkv_ctx* ctx) {
     if (!ctx) return SHOTKV_ERR_INVALID_ARG;
     CUDA_TRY(ctx, cudaSetDevice(ctx->device));
+    if (ctx->err_host && *(volatile int*)ctx->err_host) {
+        *(volatile int*)ctx->err_host = 0;
+        return fail(ctx, SHOTKV_ERR_TIMEOUT, "an earlier scoring kernel gave up a bounded wait; its outputs are invalid");
+    }
     return SHOTKV_OK;
+}
+
+// ---- tensor-core scoring: tensor maps and launch ----------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+template <int D, int MB>
+int launch_score_tc_t(shotkv_ctx* ctx, const CUtensorMap& tmQ, const CUtensorMap& tmK, int qbox, int kbox,
+                      const ScoreTcParams& sp, cudaStream_t stream) {
+    constexpr int smem = ScoreTcCfg<D, MB>::kSmemBytes;
+    CUDA_TRY(ctx, cudaFuncSetAttribute(score_tc_kernel<D, MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    int grid = sp.total_items < ctx->sm_count ? sp.total_items : ctx->sm_count;
+    if (grid < 1) grid = 1;
+    score_tc_kernel<D, MB><<<grid, 384, smem, stream>>>(tmQ, tmK, qbox, kbox, sp);
+    LAUNCH_CHECK(ctx);
+    return SHOTKV_OK;
+}
+
+int launch_score_tc(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const shotkv_bf16* K, const PrefillWs& w,
+                    int P, cudaStream_t stream) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return fail(ctx, SHOTKV_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+    if (((uintptr_t)Q | (uintptr_t)K) & 15) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "Qwin and K must be 16-byte aligned");
+    const long long U = (long long)d->B * d->L * d->Hkv;
+    const int R = (d->H / d->Hkv) * d->W;
+    const long long qrows = U * R;
+    const int qbox = qrows < 128 ? (int)qrows : 128, kbox = d->N < 128 ? d->N : 128;
+    CUtensorMap tmQ, tmK;
+    {
+        cuuint64_t dims[2] = {(cuuint64_t)d->d, (cuuint64_t)qrows};
+        cuuint64_t strides[1] = {(cuuint64_t)d->d * 2};
+        cuuint32_t box[2] = {64, (cuuint32_t)qbox}, es[2] = {1, 1};
+        CUresult r = enc(&tmQ, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)Q, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail(ctx, SHOTKV_ERR_CUDA, "cuTensorMapEncodeTiled(Qwin) failed with %d", (int)r);
+    }
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)d->d, (cuuint64_t)d->N, (cuuint64_t)U};
+        cuuint64_t strides[2] = {(cuuint64_t)d->d * 2, (cuuint64_t)d->N * d->d * 2};
+        cuuint32_t box[3] = {64, (cuuint32_t)kbox, 1}, es[3] = {1, 1, 1};
+        CUresult r = enc(&tmK, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)K, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail(ctx, SHOTKV_ERR_CUDA, "cuTensorMapEncodeTiled(K) failed with %d", (int)r);
+    }
+    ScoreTcParams sp{};
+    sp.pieces = w.pieces;
+    sp.P = P;
+    sp.L = d->L; sp.Hkv = d->Hkv; sp.N = d->N; sp.W = d->W; sp.R = R; sp.Rpad = rpad_of(d);
+    if (U * P > 0x7fffffffLL) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "too many work items");
+    sp.total_items = (int)(U * P);
+    sp.scale_log2 = kLog2e / sqrtf((float)d->d);
+    sp.part_m = w.part_m; sp.part_z = w.part_z;
+    sp.err = ctx->err_dev;
+    const bool big = sp.Rpad == 256;
+    if (d->d == 128) return big ? launch_score_tc_t<128, 2>(ctx, tmQ, tmK, qbox, kbox, sp, stream) : launch_score_tc_t<128, 1>(ctx, tmQ, tmK, qbox, kbox, sp, stream);
+    return big ? launch_score_tc_t<64, 2>(ctx, tmQ, tmK, qbox, kbox, sp, stream) : launch_score_tc_t<64, 1>(ctx, tmQ, tmK, qbox, kbox, sp, stream);
 }
 
 int check_ws(shotkv_ctx* ctx, const shotkv_dims* d, void* ws, size_t ws_bytes) {
@@ -285,7 +364,8 @@ int run_stats(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const
     const int U = d->B * d->L * d->Hkv;
     ScoreParams sp = base_params(d, Q, K, w, P);
     prof_mark(ctx, stream);
-    rc = launch_score<false>(ctx, d, sp, U, stream);
+    static const bool use_mma = getenv("SHOTKV_SCORE_MMA") != nullptr;      // development A/B switch
+    rc = use_mma ? launch_score<false>(ctx, d, sp, U, stream) : launch_score_tc(ctx, d, Q, K, w, P, stream);
     if (rc) return rc;
     if (need_rows) {
         row_stats_kernel<<<U, 256, 0, stream>>>(w.part_m, w.part_z, P, sp.R, sp.Rpad, w.row_m, w.row_invz);
@@ -353,6 +433,13 @@ int shotkv_create(shotkv_ctx** out, int device) {
             delete ctx;
             return SHOTKV_ERR_CUDA;
         }
+    if (cudaHostAlloc((void**)&ctx->err_host, sizeof(int), cudaHostAllocMapped) != cudaSuccess ||
+        cudaHostGetDevicePointer((void**)&ctx->err_dev, ctx->err_host, 0) != cudaSuccess) {
+        shotkv_destroy(ctx);
+        return SHOTKV_ERR_CUDA;
+    }
+    *ctx->err_host = 0;
+    ctx->sm_count = prop.multiProcessorCount;
     *out = ctx;
     return SHOTKV_OK;
 }
@@ -366,6 +453,7 @@ void shotkv_destroy(shotkv_ctx* ctx) {
             cudaEventDestroy(ctx->stage_done[i]);
         }
     if (ctx->stage) cudaFreeHost(ctx->stage);
+    if (ctx->err_host) cudaFreeHost(ctx->err_host);
     for (int i = 0; i < kProfSlots; ++i)
         for (int j = 0; j < 4; ++j)
             if (ctx->prof_ev[i][j]) cudaEventDestroy(ctx->prof_ev[i][j]);
