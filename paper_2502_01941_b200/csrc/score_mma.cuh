@@ -236,9 +236,12 @@ __global__ void __launch_bounds__(256, (MB == 1 ? 2 : 1)) score_mma_kernel(const
 
 // Per (unit, row): m = max over pieces, Z = sum z_p * exp2(m_p - m); stores m and 1/Z
 // (0 for padding rows).  Fixed piece order, so the result does not depend on scheduling.
-__global__ void row_stats_kernel(const float* __restrict__ part_m, const float* __restrict__ part_z, int P, int R,
+// Pieces whose segment id is above `last_seg` are list padding and are skipped.
+__global__ void row_stats_kernel(const float* __restrict__ part_m, const float* __restrict__ part_z,
+                                 const int* __restrict__ piece_seg, int units_per_prompt, int last_seg, int P, int R,
                                  int Rpad, float* __restrict__ row_m, float* __restrict__ row_invz) {
     const int u = blockIdx.x;
+    const int* seg = piece_seg + (size_t)(u / units_per_prompt) * P;
     for (int r = threadIdx.x; r < Rpad; r += blockDim.x) {
         if (r >= R) {   // padding rows carry no weight; their partials may be anything
             row_m[(size_t)u * Rpad + r] = 0.f;
@@ -248,11 +251,13 @@ __global__ void row_stats_kernel(const float* __restrict__ part_m, const float* 
         const float* pm = part_m + (size_t)u * P * Rpad + r;
         const float* pz = part_z + (size_t)u * P * Rpad + r;
         float m = SHOTKV_NEG_INF;
-        for (int q = 0; q < P; ++q) m = fmaxf(m, pm[(size_t)q * Rpad]);
+        for (int q = 0; q < P; ++q)
+            if (seg[q] <= last_seg) m = fmaxf(m, pm[(size_t)q * Rpad]);
         float z = 0.f;
-        for (int q = 0; q < P; ++q) z += pz[(size_t)q * Rpad] * ex2f(pm[(size_t)q * Rpad] - m);
+        for (int q = 0; q < P; ++q)
+            if (seg[q] <= last_seg) z += pz[(size_t)q * Rpad] * ex2f(pm[(size_t)q * Rpad] - m);
         row_m[(size_t)u * Rpad + r] = m;
-        row_invz[(size_t)u * Rpad + r] = (r < R && z > 0.f) ? 1.f / z : 0.f;
+        row_invz[(size_t)u * Rpad + r] = z > 0.f ? 1.f / z : 0.f;
     }
 }
 
@@ -275,8 +280,10 @@ __global__ void __launch_bounds__(THREADS) shot_mass_kernel(const float* __restr
     const bool live = r < R;
     float m = SHOTKV_NEG_INF, z = 0.f;
     if (live) {
-        for (int q = 0; q < P; ++q) m = fmaxf(m, pm[(size_t)q * Rpad]);
-        for (int q = 0; q < P; ++q) z += pz[(size_t)q * Rpad] * ex2f(pm[(size_t)q * Rpad] - m);
+        for (int q = 0; q < P; ++q)
+            if (seg[q] <= S + 1) m = fmaxf(m, pm[(size_t)q * Rpad]);      // ids above S+1 are list padding
+        for (int q = 0; q < P; ++q)
+            if (seg[q] <= S + 1) z += pz[(size_t)q * Rpad] * ex2f(pm[(size_t)q * Rpad] - m);
     }
     const float invz = (live && z > 0.f) ? 1.f / z : 0.f;
     int q = 0;

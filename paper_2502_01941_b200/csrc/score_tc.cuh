@@ -1,18 +1,23 @@
 // Window attention scoring on the 5th-generation tensor cores (tcgen05.mma, accumulators in
 // tensor memory) with K streamed by TMA: the STATS pass of the scoring step.
 //
-// Persistent CTAs, one per SM, each owning a contiguous range of (unit, piece) work items
-// (unit = prompt x layer x kv head; a piece is a key range of at most 512 keys that never
-// straddles a shot boundary).  Warp roles:
+// Persistent CTAs, one per SM, each owning a contiguous range of work items.  An item is one
+// (unit, chunk): unit = prompt x layer x kv head, chunk = a run of whole 128-key tiles of that
+// unit's keys.  Chunk ends and shot boundaries cut the keys into "pieces"; per (piece, window
+// row) the kernel emits a reference maximum m and z = sum exp2(x - m) over the piece's keys.
+// Warp roles:
 //   warp 0      TMA producer: the unit's window queries Q (once per unit) and K tiles of 128 keys
 //               into a ring of 128-byte-swizzled shared-memory stages
 //   warp 1      MMA issuer: S[128 x 128] = Q_block . K_tile^T per 128-row block of Q, fp32
 //               accumulators double-buffered in tensor memory
 //   warp 2      tensor-memory allocation
-//   warps 4-11  epilogue: one thread per window row; reads its row of S from tensor memory and
-//               keeps, per piece, a reference maximum m and z = sum exp2(x - m)
-// Per (piece, row) the pair (m, z) goes to global memory; the reductions over pieces, rows and
-// heads that turn them into shot scores are done by the kernels in score_mma.cuh.
+//   warps 4-19  epilogue: every thread owns one window row and a slice of a tile's columns (64
+//               of 128 when there are two row blocks, 32 when there is one), walks them in
+//               chunks of 32 registers, and splits its running sum wherever a piece ends inside
+//               a chunk.  The slices of a row are merged through shared memory when a piece is
+//               complete, in a fixed order.
+// The reductions over pieces, rows and heads that turn (m, z) into shot scores are done by the
+// kernels in score_mma.cuh.
 //
 // Every wait on an mbarrier is bounded: after about two seconds a waiter raises the CTA's abort
 // flag and the device error word, all roles leave their loops, outstanding bulk copies are
@@ -25,10 +30,13 @@
 namespace shotkv {
 
 struct ScoreTcParams {
-    const int2* pieces;   // [B][P] key ranges [lo, hi)
-    int P;                // pieces per prompt
+    const int2* pieces;       // [B][P] key ranges [lo, hi), ascending, covering [0, N)
+    const int* chunk_first;   // [B][cf_stride] index of the first piece of every chunk (nchunk + 1 used)
+    int cf_stride;
+    int P;                    // pieces per prompt (row length of `pieces`)
+    int nchunk, chunk_keys;   // chunks per unit; keys per chunk (a multiple of 128)
     int L, Hkv, N, W, R, Rpad;
-    int total_items;      // U * P
+    int total_items;          // U * nchunk
     float scale_log2;     // log2(e)/sqrt(d)
     float* part_m;        // [U][P][Rpad]
     float* part_z;        // [U][P][Rpad]
@@ -43,7 +51,10 @@ struct ScoreTcCfg {
     static constexpr int kStageBytes = kSub * kSubBytes;
     static constexpr int kStages = D == 128 ? (MB == 2 ? 4 : 5) : 6;
     static constexpr int kBarBytes = 1024;
-    static constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kBarBytes + 2 * 128 * 2 * 4 + 1024;
+    static constexpr int kCombBytes = 2 * 4 * 128 * 2 * 4;   // [parity][slice][row][m, z]
+    static constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kBarBytes + kCombBytes + 1024;
+    static constexpr int kSlices = 4 / MB;                    // column slices of a tile, one per epilogue warpgroup
+    static constexpr int kThreads = 128 + 16 * 32;
 };
 
 namespace tc {
@@ -158,50 +169,39 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[32]) {
                  : "memory");
 }
 
-// One 32-column chunk of a row: mask, refresh the reference maximum if the chunk exceeds it by
-// more than 2^8, add exp2(x*scale - m) to the running sum.  `valid` = columns of the chunk that
-// count (<= 0: none, >= 32: all).
-__device__ __forceinline__ void row_chunk(uint32_t (&raw)[32], int valid, float scale, float& m_ref, float& z) {
-    float v[32];
+// Sum of e[i] for i in [a, b) with compile-time register indices.
+__device__ __forceinline__ float range_sum(const uint32_t (&e)[32], int a, int b) {
+    float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(raw[i]);
-    if (!__all_sync(0xffffffffu, valid >= 32)) {
-#pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = i < valid ? v[i] : SHOTKV_NEG_INF;
+    for (int i = 0; i < 32; i += 2) {
+        s0 += (i >= a && i < b) ? __uint_as_float(e[i]) : 0.f;
+        s1 += (i + 1 >= a && i + 1 < b) ? __uint_as_float(e[i + 1]) : 0.f;
     }
-    float c0 = fmaxf(v[0], v[1]), c1 = fmaxf(v[2], v[3]), c2 = fmaxf(v[4], v[5]), c3 = fmaxf(v[6], v[7]);
+    return s0 + s1;
+}
+
+__device__ __forceinline__ float chunk_max(const uint32_t (&r)[32]) {
+    float c0 = fmaxf(__uint_as_float(r[0]), __uint_as_float(r[1])), c1 = fmaxf(__uint_as_float(r[2]), __uint_as_float(r[3]));
+    float c2 = fmaxf(__uint_as_float(r[4]), __uint_as_float(r[5])), c3 = fmaxf(__uint_as_float(r[6]), __uint_as_float(r[7]));
 #pragma unroll
     for (int i = 8; i < 32; i += 8) {
-        c0 = fmaxf(c0, fmaxf(v[i], v[i + 1]));
-        c1 = fmaxf(c1, fmaxf(v[i + 2], v[i + 3]));
-        c2 = fmaxf(c2, fmaxf(v[i + 4], v[i + 5]));
-        c3 = fmaxf(c3, fmaxf(v[i + 6], v[i + 7]));
+        c0 = fmaxf(c0, fmaxf(__uint_as_float(r[i]), __uint_as_float(r[i + 1])));
+        c1 = fmaxf(c1, fmaxf(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])));
+        c2 = fmaxf(c2, fmaxf(__uint_as_float(r[i + 4]), __uint_as_float(r[i + 5])));
+        c3 = fmaxf(c3, fmaxf(__uint_as_float(r[i + 6]), __uint_as_float(r[i + 7])));
     }
-    const float cm = fmaxf(fmaxf(c0, c1), fmaxf(c2, c3)) * scale;
-    if (cm > m_ref + 8.f) {            // also taken the first time (m_ref = -inf, z = 0)
-        z *= ex2f(m_ref - cm);
-        m_ref = cm;
-    }
-    const float neg = m_ref == SHOTKV_NEG_INF ? 0.f : -m_ref;
-    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-    for (int i = 0; i < 32; i += 4) {
-        s0 += ex2f(fmaf(v[i], scale, neg));
-        s1 += ex2f(fmaf(v[i + 1], scale, neg));
-        s2 += ex2f(fmaf(v[i + 2], scale, neg));
-        s3 += ex2f(fmaf(v[i + 3], scale, neg));
-    }
-    z += (s0 + s1) + (s2 + s3);
+    return fmaxf(fmaxf(c0, c1), fmaxf(c2, c3));
 }
 
 }  // namespace tc
 
 template <int D, int MB>
-__global__ void __launch_bounds__(384, 1) score_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
-                                                         const __grid_constant__ CUtensorMap tmK, const int q_box_rows,
-                                                         const int k_box_rows, const ScoreTcParams p) {
+__global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
+    score_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const int q_box_rows,
+                    const int k_box_rows, const ScoreTcParams p) {
     using Cfg = ScoreTcCfg<D, MB>;
     constexpr int NSUB = Cfg::kSub, KSTEPS = D / 16, NST = Cfg::kStages, TN = tc::kTileKeys;
+    constexpr int NSL = Cfg::kSlices, SLW = TN / NSL, NCH = SLW / 32;     // slices, slice width, chunks per slice
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;
@@ -215,7 +215,7 @@ __global__ void __launch_bounds__(384, 1) score_tc_kernel(const __grid_constant_
     const uint32_t tmem_slot = sBar + 8u * (2 * NST + 6);
     volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(gbase + (tmem_slot - base));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + (tmem_slot - base) + 4);
-    float* comb = reinterpret_cast<float*>(gbase + (sBar - base) + Cfg::kBarBytes);   // [2][128][2], MB == 1 only
+    float* comb = reinterpret_cast<float*>(gbase + (sBar - base) + Cfg::kBarBytes);   // [2][4][128][2]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -228,7 +228,7 @@ __global__ void __launch_bounds__(384, 1) score_tc_kernel(const __grid_constant_
         tc::mbar_init(bar_qempty, 1);
         for (int a = 0; a < 2; ++a) {
             tc::mbar_init(bar_tfull(a), 1);
-            tc::mbar_init(bar_tempty(a), 8);      // one arrival per epilogue warp
+            tc::mbar_init(bar_tempty(a), 16);     // one arrival per epilogue warp
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -245,7 +245,6 @@ __global__ void __launch_bounds__(384, 1) score_tc_kernel(const __grid_constant_
     const long long total = p.total_items;
     const int item_begin = (int)(total * blockIdx.x / gridDim.x);
     const int item_end = (int)(total * (blockIdx.x + 1) / gridDim.x);
-    const int units_per_prompt = p.L * p.Hkv;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -254,19 +253,19 @@ __global__ void __launch_bounds__(384, 1) score_tc_kernel(const __grid_constant_
             uint32_t ephase = 1, qephase = 1;
             bool ok = true;
             for (int it = item_begin; it < item_end && ok; ++it) {
-                const int u = it / p.P, pc = it - u * p.P;
-                const int2 r = p.pieces[(size_t)(u / units_per_prompt) * p.P + pc];
-                const int nt = (r.y - r.x + TN - 1) / TN;
+                const int u = it / p.nchunk, j = it - u * p.nchunk;
+                const int lo = j * p.chunk_keys, hi = min(p.N, lo + p.chunk_keys);
+                const int nt = (hi - lo + TN - 1) / TN;
                 if (nt <= 0) continue;
                 if (u != cur_u) {
                     if (!(ok = tc::mbar_wait(bar_qempty, qephase, abort_flag, p.err))) break;
                     qephase ^= 1;
                     tc::mbar_expect_tx(bar_qfull, MB * NSUB * q_box_rows * 128);
 #pragma unroll
-                    for (int j = 0; j < MB; ++j)
+                    for (int b = 0; b < MB; ++b)
 #pragma unroll
                         for (int sub = 0; sub < NSUB; ++sub)
-                            tc::tma_load_2d(sQ + (j * NSUB + sub) * Cfg::kSubBytes, &tmQ, sub * 64, u * p.R + j * 128, bar_qfull);
+                            tc::tma_load_2d(sQ + (b * NSUB + sub) * Cfg::kSubBytes, &tmQ, sub * 64, u * p.R + b * 128, bar_qfull);
                     cur_u = u;
                 }
                 for (int t = 0; t < nt; ++t) {
@@ -274,7 +273,7 @@ __global__ void __launch_bounds__(384, 1) score_tc_kernel(const __grid_constant_
                     tc::mbar_expect_tx(bar_full(stage), NSUB * k_box_rows * 128);
 #pragma unroll
                     for (int sub = 0; sub < NSUB; ++sub)
-                        tc::tma_load_3d(sK + stage * Cfg::kStageBytes + sub * Cfg::kSubBytes, &tmK, sub * 64, r.x + t * TN, u,
+                        tc::tma_load_3d(sK + stage * Cfg::kStageBytes + sub * Cfg::kSubBytes, &tmK, sub * 64, lo + t * TN, u,
                                         bar_full(stage));
                     outstanding = outstanding < NST ? outstanding + 1 : NST;
                     if (++stage == NST) {
@@ -303,12 +302,12 @@ __global__ void __launch_bounds__(384, 1) score_tc_kernel(const __grid_constant_
         if (lane == 0) {
             constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TN >> 3) << 17) | ((128u >> 4) << 24);
             int stage = 0, acc = 0, cur_u = -1;
-            uint32_t fphase = 0, qfphase = 0, tephase[2] = {1, 1};
+            uint32_t fphase = 0, qfphase = 0, tephase0 = 1, tephase1 = 1;
             bool ok = true;
             for (int it = item_begin; it < item_end && ok; ++it) {
-                const int u = it / p.P, pc = it - u * p.P;
-                const int2 r = p.pieces[(size_t)(u / units_per_prompt) * p.P + pc];
-                const int nt = (r.y - r.x + TN - 1) / TN;
+                const int u = it / p.nchunk, j = it - u * p.nchunk;
+                const int lo = j * p.chunk_keys, hi = min(p.N, lo + p.chunk_keys);
+                const int nt = (hi - lo + TN - 1) / TN;
                 if (nt <= 0) continue;
                 if (u != cur_u) {
                     if (cur_u >= 0) tc::umma_commit(bar_qempty);     // Q may be replaced once these MMAs are done
@@ -318,16 +317,17 @@ __global__ void __launch_bounds__(384, 1) score_tc_kernel(const __grid_constant_
                 }
                 for (int t = 0; t < nt; ++t) {
                     if (!(ok = tc::mbar_wait(bar_full(stage), fphase, abort_flag, p.err))) break;
-                    if (!(ok = tc::mbar_wait(bar_tempty(acc), tephase[acc], abort_flag, p.err))) break;
-                    tephase[acc] ^= 1;
+                    const uint32_t tph = acc ? tephase1 : tephase0;
+                    if (!(ok = tc::mbar_wait(bar_tempty(acc), tph, abort_flag, p.err))) break;
+                    if (acc) tephase1 ^= 1; else tephase0 ^= 1;
                     tc::fence_after_sync();
                     const uint32_t kb = sK + stage * Cfg::kStageBytes;
 #pragma unroll
-                    for (int j = 0; j < MB; ++j) {
-                        const uint32_t d_tmem = tmem_base + (uint32_t)((acc * MB + j) * TN);
+                    for (int b = 0; b < MB; ++b) {
+                        const uint32_t d_tmem = tmem_base + (uint32_t)((acc * MB + b) * TN);
 #pragma unroll
                         for (int ks = 0; ks < KSTEPS; ++ks) {
-                            const uint32_t a_addr = sQ + (j * NSUB + (ks >> 2)) * Cfg::kSubBytes + (ks & 3) * 32;
+                            const uint32_t a_addr = sQ + (b * NSUB + (ks >> 2)) * Cfg::kSubBytes + (ks & 3) * 32;
                             const uint32_t b_addr = kb + (ks >> 2) * Cfg::kSubBytes + (ks & 3) * 32;
                             tc::umma_bf16(d_tmem, tc::smem_desc(a_addr), tc::smem_desc(b_addr), idesc, ks > 0);
                         }
@@ -344,73 +344,133 @@ __global__ void __launch_bounds__(384, 1) score_tc_kernel(const __grid_constant_
         }
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ epilogue
-        const int wg = (warp - 4) >> 2, quad = warp & 3;
-        const int blk = MB == 2 ? wg : 0;                 // 128-row block of Q this warpgroup reads
-        const int col_base = MB == 2 ? 0 : wg * 64;       // MB == 1: the two warpgroups split the columns
-        constexpr int NCH = MB == 2 ? 4 : 2;
-        const int row = blk * 128 + quad * 32 + lane;
+        const int g = (warp - 4) >> 2, quad = warp & 3;
+        const int blk = MB == 2 ? (g >> 1) : 0;            // 128-row block of Q
+        const int slice = MB == 2 ? (g & 1) : g;           // column slice of every tile
+        const int lrow = quad * 32 + lane;
+        const int row = blk * 128 + lrow;
         const int plim = row < p.R ? p.N - p.W + (row % p.W) : p.N - 1;
-        int acc = 0, item_no = 0;
-        uint32_t tfphase[2] = {0, 0};
+        const float scale = p.scale_log2;
+        const int units_per_prompt = p.L * p.Hkv;
+        int acc = 0, nflush = 0;
+        uint32_t tfphase0 = 0, tfphase1 = 0;
         bool ok = true;
-        for (int it = item_begin; it < item_end && ok; ++it, ++item_no) {
-            const int u = it / p.P, pc = it - u * p.P;
-            const int2 r = p.pieces[(size_t)(u / units_per_prompt) * p.P + pc];
-            const int nt = (r.y - r.x + TN - 1) / TN;
+        for (int it = item_begin; it < item_end && ok; ++it) {
+            const int u = it / p.nchunk, j = it - u * p.nchunk;
+            const int lo = j * p.chunk_keys, hi = min(p.N, lo + p.chunk_keys);
+            const int nt = (hi - lo + TN - 1) / TN;
+            const int bprompt = u / units_per_prompt;
+            const int2* pcs = p.pieces + (size_t)bprompt * p.P;
+            int pi = p.chunk_first[(size_t)bprompt * p.cf_stride + j];
+            const int pi_last = p.chunk_first[(size_t)bprompt * p.cf_stride + j + 1];
+            int pend = pi < pi_last ? pcs[pi].y : 0x7fffffff;
             float m_ref = SHOTKV_NEG_INF, z = 0.f;
+
+            // piece `pi` is complete for this thread's columns: merge the row's slices, write, move on
+            auto flush = [&]() {
+                // slot of warpgroup g' and local row r: comb[parity][g'][r][m, z]; a row's slices are the
+                // NSL consecutive warpgroups starting at its leader (slice 0)
+                float* slot = comb + (nflush & 1) * 1024 + (g - slice) * 256 + lrow * 2;
+                if (slice != 0) {
+                    slot[slice * 256] = m_ref;
+                    slot[slice * 256 + 1] = z;
+                }
+                if (blk == 0) asm volatile("bar.sync 1, %0;" ::"n"(NSL * 128) : "memory");
+                else asm volatile("bar.sync 2, %0;" ::"n"(NSL * 128) : "memory");
+                if (slice == 0) {
+                    float mm = m_ref;
+#pragma unroll
+                    for (int s = 1; s < NSL; ++s) mm = fmaxf(mm, slot[s * 256]);
+                    const float mu = mm == SHOTKV_NEG_INF ? 0.f : mm;
+                    float zz = z * ex2f(m_ref - mu);
+#pragma unroll
+                    for (int s = 1; s < NSL; ++s) zz += slot[s * 256 + 1] * ex2f(slot[s * 256] - mu);
+                    const size_t o = ((size_t)u * p.P + pi) * p.Rpad + row;
+                    const bool live = row < p.R;        // padding rows: their Q was never loaded
+                    p.part_m[o] = live ? mm : 0.f;
+                    p.part_z[o] = live ? zz : 0.f;
+                }
+                z = 0.f;
+                ++nflush;
+                ++pi;
+                pend = pi < pi_last ? pcs[pi].y : 0x7fffffff;
+            };
+
+            // 32 columns starting at key kc0
+            auto chunk = [&](uint32_t (&raw)[32], int kc0) {
+                while (pend <= kc0) flush();
+                const int lim = min(hi, plim + 1) - kc0;               // columns of this chunk that count
+                const bool plain = __all_sync(0xffffffffu, lim >= 32) && pend >= kc0 + 32;
+                if (plain) {
+                    const float cm = tc::chunk_max(raw) * scale;
+                    if (cm > m_ref + 8.f) {
+                        z *= ex2f(m_ref - cm);
+                        m_ref = cm;
+                    }
+                    const float neg = -m_ref;
+                    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) {
+                        s0 += ex2f(fmaf(__uint_as_float(raw[i]), scale, neg));
+                        s1 += ex2f(fmaf(__uint_as_float(raw[i + 1]), scale, neg));
+                        s2 += ex2f(fmaf(__uint_as_float(raw[i + 2]), scale, neg));
+                        s3 += ex2f(fmaf(__uint_as_float(raw[i + 3]), scale, neg));
+                    }
+                    z += (s0 + s1) + (s2 + s3);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (i >= lim) raw[i] = 0xff800000u;              // -inf: beyond the chunk's end or the row's position
+                    const float cm = tc::chunk_max(raw) * scale;
+                    if (cm > m_ref + 8.f) {
+                        z *= ex2f(m_ref - cm);
+                        m_ref = cm;
+                    }
+                    const float neg = m_ref == SHOTKV_NEG_INF ? 0.f : -m_ref;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) raw[i] = __float_as_uint(ex2f(fmaf(__uint_as_float(raw[i]), scale, neg)));
+                    int start = 0;
+                    while (pend < kc0 + 32) {                            // pieces that end inside this chunk
+                        z += tc::range_sum(raw, start, pend - kc0);
+                        start = pend - kc0;
+                        flush();
+                    }
+                    z += tc::range_sum(raw, start, 32);
+                }
+            };
+
             for (int t = 0; t < nt; ++t) {
-                ok = tc::mbar_wait(bar_tfull(acc), tfphase[acc], abort_flag, p.err);
+                const uint32_t tph = acc ? tfphase1 : tfphase0;
+                ok = tc::mbar_wait(bar_tfull(acc), tph, abort_flag, p.err);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                tfphase[acc] ^= 1;
+                if (acc) tfphase1 ^= 1; else tfphase0 ^= 1;
                 tc::fence_after_sync();
-                const int key0 = r.x + t * TN;
-                const int lim = min(r.y - key0, plim + 1 - key0) - col_base;     // valid columns from col_base on
-                const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)((acc * MB + blk) * TN + col_base);
-                uint32_t va[32], vb[32];
+                const int kc0 = lo + t * TN + slice * SLW;
+                const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)((acc * MB + blk) * TN + slice * SLW);
+                uint32_t va[32];
                 tc::tmem_ld32(va, taddr);
-#pragma unroll
-                for (int c = 0; c < NCH; c += 2) {
+                if (NCH == 2) {
+                    uint32_t vb[32];
                     tc::tmem_ld_wait(va);
-                    tc::tmem_ld32(vb, taddr + (c + 1) * 32);
-                    tc::row_chunk(va, lim - c * 32, p.scale_log2, m_ref, z);
+                    tc::tmem_ld32(vb, taddr + 32);
+                    chunk(va, kc0);
                     tc::tmem_ld_wait(vb);
-                    if (c + 2 < NCH) {
-                        tc::tmem_ld32(va, taddr + (c + 2) * 32);
-                    } else {
-                        // this tile's accumulators are in registers: hand the buffer back
-                        tc::fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) tc::mbar_arrive(bar_tempty(acc));
-                    }
-                    tc::row_chunk(vb, lim - (c + 1) * 32, p.scale_log2, m_ref, z);
+                    tc::fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(bar_tempty(acc));      // accumulators are in registers
+                    chunk(vb, kc0 + 32);
+                } else {
+                    tc::tmem_ld_wait(va);
+                    tc::fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(bar_tempty(acc));
+                    chunk(va, kc0);
                 }
                 acc ^= 1;
             }
             if (!ok) break;
-            const size_t o = ((size_t)u * p.P + pc) * p.Rpad + row;
-            if (row >= p.R) {          // padding row: its Q rows were never loaded; keep the partials finite
-                m_ref = 0.f;
-                z = 0.f;
-            }
-            if (MB == 2) {
-                p.part_m[o] = m_ref;
-                p.part_z[o] = z;
-            } else {
-                float* cb = comb + (item_no & 1) * 256 + (quad * 32 + lane) * 2;
-                if (wg == 1) {
-                    cb[0] = m_ref;
-                    cb[1] = z;
-                }
-                asm volatile("bar.sync 1, 256;" ::: "memory");
-                if (wg == 0) {
-                    const float m1 = cb[0], z1 = cb[1];
-                    const float mm = fmaxf(m_ref, m1);
-                    const float mu = mm == SHOTKV_NEG_INF ? 0.f : mm;
-                    p.part_m[o] = mm;
-                    p.part_z[o] = z * ex2f(m_ref - mu) + z1 * ex2f(m1 - mu);
-                }
-            }
+            while (pi < pi_last) flush();
         }
     }
 

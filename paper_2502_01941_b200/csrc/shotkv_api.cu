@@ -22,7 +22,7 @@ using namespace shotkv;
 
 namespace {
 
-constexpr int kPieceMaxKeys = 512;     // longest key range one scoring work item covers
+constexpr int kMaxChunks = 64;         // most chunks a unit's keys are split into for load balance
 constexpr int kMaxShots = 8192;
 constexpr int kStageSlots = 4;
 constexpr size_t kStageSlotBytes = 1u << 20;
@@ -135,12 +135,13 @@ int check_offsets(const shotkv_dims* d, const shotkv_policy* p, const int32_t* o
 }
 
 int rpad_of(const shotkv_dims* d) { return (d->H / d->Hkv) * d->W <= 128 ? 128 : 256; }
-int pmax_of(const shotkv_dims* d) { return d->S + 2 + d->N / kPieceMaxKeys + 1; }
+int pmax_of(const shotkv_dims* d) { return d->S + 2 + kMaxChunks + 1; }
 
 struct PrefillWs {
     int* off;          // [B][S+1]
     int2* pieces;      // [B][Pmax]
     int* piece_seg;    // [B][Pmax]
+    int* chunk_first;  // [B][kMaxChunks + 1]
     float* part_m;     // [U][Pmax][Rpad]
     float* part_z;
     float* row_m;      // [U][Rpad]
@@ -157,6 +158,7 @@ PrefillWs carve(const shotkv_dims* d, void* base) {
     w.off = (int*)take((size_t)d->B * (d->S + 1) * 4);
     w.pieces = (int2*)take((size_t)d->B * P * 8);
     w.piece_seg = (int*)take((size_t)d->B * P * 4);
+    w.chunk_first = (int*)take((size_t)d->B * (kMaxChunks + 1) * 4);
     w.part_m = (float*)take(U * P * R * 4);
     w.part_z = (float*)take(U * P * R * 4);
     w.row_m = (float*)take(U * R * 4);
@@ -185,19 +187,54 @@ int upload_small(shotkv_ctx* ctx, void* dst, const void* src, size_t bytes, cuda
     return SHOTKV_OK;
 }
 
-// Splits [0, N) into pieces of at most kPieceMaxKeys keys.  With offsets: pieces never cross a
-// segment boundary (segment 0 = before the first shot, i+1 = shot i, S+1 = the question) and
-// piece_seg records the segment.  Without: plain fixed-size chunks.  Returns pieces per prompt
-// (padded with empty pieces to the same count for every prompt).
-int build_pieces(const shotkv_dims* d, const int32_t* off, std::vector<int2>& pieces, std::vector<int>& seg) {
+// Work partition of the scoring pass.  Every unit's keys are cut into `nchunk` chunks of
+// `chunk_keys` keys (whole 128-key tiles); an item is one (unit, chunk) and the persistent CTAs
+// take equal runs of consecutive items.  The split that minimises the busiest CTA's tile count
+// wins; each extra chunk costs one more piece per unit, so ties go to fewer chunks.
+struct ChunkPlan { int nchunk, chunk_keys; };
+ChunkPlan plan_chunks(const shotkv_dims* d, int sm_count) {
+    const long long U = (long long)d->B * d->L * d->Hkv;
+    const int tiles = (d->N + 127) / 128;
+    ChunkPlan best{1, tiles * 128};
+    long long best_cost = -1;
+    for (int want = 1; want <= kMaxChunks && want <= tiles; ++want) {
+        const int ct = (tiles + want - 1) / want;             // tiles per chunk
+        const int nchunk = (tiles + ct - 1) / ct;
+        const long long items = U * nchunk;
+        const long long ctas = items < sm_count ? items : sm_count;
+        const long long per_cta = (items + ctas - 1) / ctas;
+        const long long cost = per_cta * (ct * 16 + 3);       // a tile plus a small per-item overhead, in 1/16 tiles
+        if (best_cost < 0 || cost < best_cost) {
+            best_cost = cost;
+            best = ChunkPlan{nchunk, ct * 128};
+        }
+    }
+    return best;
+}
+
+// Cuts [0, N) of every prompt into pieces at the chunk ends and, when offsets are given, at the
+// segment boundaries (segment 0 = before the first shot, i+1 = shot i, S+1 = the question).
+// piece_seg records each piece's segment (S+2 marks list padding); chunk_first[b][j] is the index
+// of the first piece of chunk j.  Returns pieces per prompt (the same for all after padding).
+int build_pieces(const shotkv_dims* d, const int32_t* off, const ChunkPlan& plan, std::vector<int2>& pieces,
+                 std::vector<int>& seg, std::vector<int>& chunk_first) {
     std::vector<std::vector<int2>> pp(d->B);
     std::vector<std::vector<int>> ss(d->B);
+    chunk_first.assign((size_t)d->B * (kMaxChunks + 1), 0);
     size_t P = 0;
     for (int b = 0; b < d->B; ++b) {
+        int* cf = chunk_first.data() + (size_t)b * (kMaxChunks + 1);
+        int next_chunk = 0;
         auto add_range = [&](int lo, int hi, int s) {
-            for (int x = lo; x < hi; x += kPieceMaxKeys) {
-                pp[b].push_back(make_int2(x, x + kPieceMaxKeys < hi ? x + kPieceMaxKeys : hi));
+            int x = lo;
+            while (x < hi) {
+                const int j = x / plan.chunk_keys;
+                const int cend = (j + 1) * plan.chunk_keys;
+                const int y = cend < hi ? cend : hi;
+                while (next_chunk <= j) cf[next_chunk++] = (int)pp[b].size();
+                pp[b].push_back(make_int2(x, y));
                 ss[b].push_back(s);
+                x = y;
             }
         };
         if (off) {
@@ -208,9 +245,11 @@ int build_pieces(const shotkv_dims* d, const int32_t* off, std::vector<int2>& pi
         } else {
             add_range(0, d->N, 0);
         }
+        while (next_chunk <= plan.nchunk) cf[next_chunk++] = (int)pp[b].size();
         if (pp[b].size() > P) P = pp[b].size();
     }
-    pieces.assign((size_t)d->B * P, make_int2(0, 0));
+    if (P == 0) P = 1;
+    pieces.assign((size_t)d->B * P, make_int2(d->N, d->N));
     seg.assign((size_t)d->B * P, d->S + 2);
     for (int b = 0; b < d->B; ++b)
         for (size_t i = 0; i < pp[b].size(); ++i) {
@@ -296,13 +335,13 @@ int launch_score_tc_t(shotkv_ctx* ctx, const CUtensorMap& tmQ, const CUtensorMap
     CUDA_TRY(ctx, cudaFuncSetAttribute(score_tc_kernel<D, MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     int grid = sp.total_items < ctx->sm_count ? sp.total_items : ctx->sm_count;
     if (grid < 1) grid = 1;
-    score_tc_kernel<D, MB><<<grid, 384, smem, stream>>>(tmQ, tmK, qbox, kbox, sp);
+    score_tc_kernel<D, MB><<<grid, ScoreTcCfg<D, MB>::kThreads, smem, stream>>>(tmQ, tmK, qbox, kbox, sp);
     LAUNCH_CHECK(ctx);
     return SHOTKV_OK;
 }
 
 int launch_score_tc(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const shotkv_bf16* K, const PrefillWs& w,
-                    int P, cudaStream_t stream) {
+                    int P, const ChunkPlan& plan, cudaStream_t stream) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return fail(ctx, SHOTKV_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
     if (((uintptr_t)Q | (uintptr_t)K) & 15) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "Qwin and K must be 16-byte aligned");
@@ -329,10 +368,14 @@ int launch_score_tc(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q,
     }
     ScoreTcParams sp{};
     sp.pieces = w.pieces;
+    sp.chunk_first = w.chunk_first;
+    sp.cf_stride = kMaxChunks + 1;
     sp.P = P;
+    sp.nchunk = plan.nchunk;
+    sp.chunk_keys = plan.chunk_keys;
     sp.L = d->L; sp.Hkv = d->Hkv; sp.N = d->N; sp.W = d->W; sp.R = R; sp.Rpad = rpad_of(d);
-    if (U * P > 0x7fffffffLL) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "too many work items");
-    sp.total_items = (int)(U * P);
+    if (U * plan.nchunk > 0x7fffffffLL) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "too many work items");
+    sp.total_items = (int)(U * plan.nchunk);
     sp.scale_log2 = kLog2e / sqrtf((float)d->d);
     sp.part_m = w.part_m; sp.part_z = w.part_z;
     sp.err = ctx->err_dev;
@@ -354,21 +397,25 @@ int check_ws(shotkv_ctx* ctx, const shotkv_dims* d, void* ws, size_t ws_bytes) {
 int run_stats(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const shotkv_bf16* K, const PrefillWs& w,
               const int32_t* off_host, bool need_rows, int* P_out, cudaStream_t stream) {
     std::vector<int2> pieces;
-    std::vector<int> seg;
-    const int P = build_pieces(d, off_host, pieces, seg);
+    std::vector<int> seg, chunk_first;
+    const ChunkPlan plan = plan_chunks(d, ctx->sm_count);
+    const int P = build_pieces(d, off_host, plan, pieces, seg, chunk_first);
     if (P > pmax_of(d)) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "internal: piece count %d exceeds bound %d", P, pmax_of(d));
     int rc = upload_small(ctx, w.pieces, pieces.data(), pieces.size() * sizeof(int2), stream);
     if (rc) return rc;
     rc = upload_small(ctx, w.piece_seg, seg.data(), seg.size() * sizeof(int), stream);
     if (rc) return rc;
+    rc = upload_small(ctx, w.chunk_first, chunk_first.data(), chunk_first.size() * sizeof(int), stream);
+    if (rc) return rc;
     const int U = d->B * d->L * d->Hkv;
     ScoreParams sp = base_params(d, Q, K, w, P);
     prof_mark(ctx, stream);
     static const bool use_mma = getenv("SHOTKV_SCORE_MMA") != nullptr;      // development A/B switch
-    rc = use_mma ? launch_score<false>(ctx, d, sp, U, stream) : launch_score_tc(ctx, d, Q, K, w, P, stream);
+    rc = use_mma ? launch_score<false>(ctx, d, sp, U, stream) : launch_score_tc(ctx, d, Q, K, w, P, plan, stream);
     if (rc) return rc;
     if (need_rows) {
-        row_stats_kernel<<<U, 256, 0, stream>>>(w.part_m, w.part_z, P, sp.R, sp.Rpad, w.row_m, w.row_invz);
+        row_stats_kernel<<<U, 256, 0, stream>>>(w.part_m, w.part_z, w.piece_seg, d->L * d->Hkv, d->S + 1, P, sp.R, sp.Rpad,
+                                                w.row_m, w.row_invz);
         LAUNCH_CHECK(ctx);
     }
     *P_out = P;
