@@ -6,11 +6,10 @@
 // unit's keys.  Chunk ends and shot boundaries cut the keys into "pieces"; per (piece, window
 // row) the kernel emits a reference maximum m and z = sum exp2(x - m) over the piece's keys.
 // Warp roles:
-//   warp 0      TMA producer: the unit's window queries Q (once per unit) and K tiles of 128 keys
+//   warp 0      tensor-memory allocation; TMA producer: the unit's window queries Q (once per unit) and K tiles of 128 keys
 //               into a ring of 128-byte-swizzled shared-memory stages
 //   warp 1      MMA issuer: S[128 x 128] = Q_block . K_tile^T per 128-row block of Q, fp32
 //               accumulators double-buffered in tensor memory
-//   warp 2      tensor-memory allocation
 //   warps 4-19  epilogue: every thread owns one window row and a slice of a tile's columns (64
 //               of 128 when there are two row blocks, 32 when there is one), walks them in
 //               chunks of 32 registers, and splits its running sum wherever a piece ends inside
@@ -54,7 +53,7 @@ struct ScoreTcCfg {
     static constexpr int kCombBytes = 2 * 4 * 128 * 2 * 4;   // [parity][slice][row][m, z]
     static constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kBarBytes + kCombBytes + 1024;
     static constexpr int kSlices = 4 / MB;                    // column slices of a tile, one per epilogue warpgroup
-    static constexpr int kThreads = 128 + 16 * 32;
+    static constexpr int kThreads = 128 + 16 * 32;            // producer, MMA issuer, two idle warps; 16 epilogue warps
 };
 
 namespace tc {
@@ -169,28 +168,76 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[32]) {
                  : "memory");
 }
 
-// Sum of e[i] for i in [a, b) with compile-time register indices.
-__device__ __forceinline__ float range_sum(const uint32_t (&e)[32], int a, int b) {
+// ---- per-row arithmetic on 32 accumulator columns held in registers -----------------------
+#define SKV_F(r, i) __uint_as_float((r)[i])
+
+__device__ __forceinline__ float max32(const uint32_t (&r)[32]) {
+    float c0 = fmaxf(SKV_F(r, 0), SKV_F(r, 1)), c1 = fmaxf(SKV_F(r, 2), SKV_F(r, 3));
+    float c2 = fmaxf(SKV_F(r, 4), SKV_F(r, 5)), c3 = fmaxf(SKV_F(r, 6), SKV_F(r, 7));
+#pragma unroll
+    for (int i = 8; i < 32; i += 8) {
+        c0 = fmaxf(c0, fmaxf(SKV_F(r, i), SKV_F(r, i + 1)));
+        c1 = fmaxf(c1, fmaxf(SKV_F(r, i + 2), SKV_F(r, i + 3)));
+        c2 = fmaxf(c2, fmaxf(SKV_F(r, i + 4), SKV_F(r, i + 5)));
+        c3 = fmaxf(c3, fmaxf(SKV_F(r, i + 6), SKV_F(r, i + 7)));
+    }
+    return fmaxf(fmaxf(c0, c1), fmaxf(c2, c3));
+}
+// columns at or beyond `valid` become -inf
+__device__ __forceinline__ void mask32(uint32_t (&r)[32], int valid) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+        if (i >= valid) r[i] = 0xff800000u;
+}
+// sum of exp2(x*scale + neg)
+__device__ __forceinline__ float expsum32(const uint32_t (&r)[32], float scale, float neg) {
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+        s0 += ex2f(fmaf(SKV_F(r, i), scale, neg));
+        s1 += ex2f(fmaf(SKV_F(r, i + 1), scale, neg));
+        s2 += ex2f(fmaf(SKV_F(r, i + 2), scale, neg));
+        s3 += ex2f(fmaf(SKV_F(r, i + 3), scale, neg));
+    }
+    return (s0 + s1) + (s2 + s3);
+}
+// exp2(x*scale + neg) in place
+__device__ __forceinline__ void exp32(uint32_t (&r)[32], float scale, float neg) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(ex2f(fmaf(SKV_F(r, i), scale, neg)));
+}
+__device__ __forceinline__ float sum32(const uint32_t (&e)[32]) {
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+        s0 += SKV_F(e, i);
+        s1 += SKV_F(e, i + 1);
+        s2 += SKV_F(e, i + 2);
+        s3 += SKV_F(e, i + 3);
+    }
+    return (s0 + s1) + (s2 + s3);
+}
+// lo = sum of e[i] for i < nb, hi = the rest (both summed directly: no subtraction of prefixes,
+// so a tiny piece next to a dominant key keeps its own relative accuracy)
+__device__ __forceinline__ void split32(const uint32_t (&e)[32], int nb, float& lo, float& hi) {
+    float l0 = 0.f, l1 = 0.f, h0 = 0.f, h1 = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        if (i < nb) l0 += SKV_F(e, i); else h0 += SKV_F(e, i);
+        if (i + 1 < nb) l1 += SKV_F(e, i + 1); else h1 += SKV_F(e, i + 1);
+    }
+    lo = l0 + l1;
+    hi = h0 + h1;
+}
+// sum of e[i] for a <= i < b
+__device__ __forceinline__ float range32(const uint32_t (&e)[32], int a, int b) {
     float s0 = 0.f, s1 = 0.f;
 #pragma unroll
     for (int i = 0; i < 32; i += 2) {
-        s0 += (i >= a && i < b) ? __uint_as_float(e[i]) : 0.f;
-        s1 += (i + 1 >= a && i + 1 < b) ? __uint_as_float(e[i + 1]) : 0.f;
+        s0 += (i >= a && i < b) ? SKV_F(e, i) : 0.f;
+        s1 += (i + 1 >= a && i + 1 < b) ? SKV_F(e, i + 1) : 0.f;
     }
     return s0 + s1;
-}
-
-__device__ __forceinline__ float chunk_max(const uint32_t (&r)[32]) {
-    float c0 = fmaxf(__uint_as_float(r[0]), __uint_as_float(r[1])), c1 = fmaxf(__uint_as_float(r[2]), __uint_as_float(r[3]));
-    float c2 = fmaxf(__uint_as_float(r[4]), __uint_as_float(r[5])), c3 = fmaxf(__uint_as_float(r[6]), __uint_as_float(r[7]));
-#pragma unroll
-    for (int i = 8; i < 32; i += 8) {
-        c0 = fmaxf(c0, fmaxf(__uint_as_float(r[i]), __uint_as_float(r[i + 1])));
-        c1 = fmaxf(c1, fmaxf(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])));
-        c2 = fmaxf(c2, fmaxf(__uint_as_float(r[i + 4]), __uint_as_float(r[i + 5])));
-        c3 = fmaxf(c3, fmaxf(__uint_as_float(r[i + 6]), __uint_as_float(r[i + 7])));
-    }
-    return fmaxf(fmaxf(c0, c1), fmaxf(c2, c3));
 }
 
 }  // namespace tc
@@ -233,7 +280,7 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 2) {
+    if (warp == 0) {
         tc::tmem_alloc(tmem_slot, 512);
         tc::tmem_relinquish();
     }
@@ -344,6 +391,8 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
         }
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ epilogue
+        // a warp may touch the 32 tensor-memory lanes given by its index modulo 4; any four
+        // consecutive warps cover all 128 rows of a block
         const int g = (warp - 4) >> 2, quad = warp & 3;
         const int blk = MB == 2 ? (g >> 1) : 0;            // 128-row block of Q
         const int slice = MB == 2 ? (g & 1) : g;           // column slice of every tile
@@ -396,46 +445,38 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
                 pend = pi < pi_last ? pcs[pi].y : 0x7fffffff;
             };
 
-            // 32 columns starting at key kc0
-            auto chunk = [&](uint32_t (&raw)[32], int kc0) {
+            // 32 columns of this thread's row, starting at key kc0
+            auto chunk = [&](uint32_t (&r)[32], int kc0) {
                 while (pend <= kc0) flush();
-                const int lim = min(hi, plim + 1) - kc0;               // columns of this chunk that count
-                const bool plain = __all_sync(0xffffffffu, lim >= 32) && pend >= kc0 + 32;
-                if (plain) {
-                    const float cm = tc::chunk_max(raw) * scale;
-                    if (cm > m_ref + 8.f) {
-                        z *= ex2f(m_ref - cm);
-                        m_ref = cm;
-                    }
-                    const float neg = -m_ref;
-                    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        s0 += ex2f(fmaf(__uint_as_float(raw[i]), scale, neg));
-                        s1 += ex2f(fmaf(__uint_as_float(raw[i + 1]), scale, neg));
-                        s2 += ex2f(fmaf(__uint_as_float(raw[i + 2]), scale, neg));
-                        s3 += ex2f(fmaf(__uint_as_float(raw[i + 3]), scale, neg));
-                    }
-                    z += (s0 + s1) + (s2 + s3);
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (i >= lim) raw[i] = 0xff800000u;              // -inf: beyond the chunk's end or the row's position
-                    const float cm = tc::chunk_max(raw) * scale;
-                    if (cm > m_ref + 8.f) {
-                        z *= ex2f(m_ref - cm);
-                        m_ref = cm;
-                    }
-                    const float neg = m_ref == SHOTKV_NEG_INF ? 0.f : -m_ref;
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) raw[i] = __float_as_uint(ex2f(fmaf(__uint_as_float(raw[i]), scale, neg)));
+                const int lim = min(hi, plim + 1) - kc0;                 // columns of the chunk that count
+                if (!__all_sync(0xffffffffu, lim >= 32)) tc::mask32(r, lim);   // end of the keys, or the causal window
+                const float cm = tc::max32(r) * scale;
+                if (cm > m_ref + 8.f) {                                   // also the first time (m_ref = -inf, z = 0)
+                    z *= ex2f(m_ref - cm);
+                    m_ref = cm;
+                }
+                const float neg = m_ref == SHOTKV_NEG_INF ? 0.f : -m_ref;
+                if (pend >= kc0 + 32) {                                   // no piece ends inside the chunk
+                    z += tc::expsum32(r, scale, neg);
+                    return;
+                }
+                tc::exp32(r, scale, neg);
+                const int pend2 = pi + 1 < pi_last ? pcs[pi + 1].y : 0x7fffffff;
+                if (pend2 >= kc0 + 32) {                                  // exactly one boundary: one predicated pass
+                    float lo_s, hi_s;
+                    tc::split32(r, pend - kc0, lo_s, hi_s);
+                    z += lo_s;
+                    flush();
+                    z = hi_s;
+                } else {                                                  // several short pieces: general walk
                     int start = 0;
-                    while (pend < kc0 + 32) {                            // pieces that end inside this chunk
-                        z += tc::range_sum(raw, start, pend - kc0);
-                        start = pend - kc0;
+                    while (pend < kc0 + 32) {
+                        const int e = pend - kc0;
+                        z += tc::range32(r, start, e);
+                        start = e;
                         flush();
                     }
-                    z += tc::range_sum(raw, start, 32);
+                    z += tc::range32(r, start, 32);
                 }
             };
 
@@ -448,24 +489,17 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
                 tc::fence_after_sync();
                 const int kc0 = lo + t * TN + slice * SLW;
                 const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)((acc * MB + blk) * TN + slice * SLW);
-                uint32_t va[32];
-                tc::tmem_ld32(va, taddr);
-                if (NCH == 2) {
-                    uint32_t vb[32];
-                    tc::tmem_ld_wait(va);
-                    tc::tmem_ld32(vb, taddr + 32);
-                    chunk(va, kc0);
-                    tc::tmem_ld_wait(vb);
-                    tc::fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) tc::mbar_arrive(bar_tempty(acc));      // accumulators are in registers
-                    chunk(vb, kc0 + 32);
-                } else {
-                    tc::tmem_ld_wait(va);
-                    tc::fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) tc::mbar_arrive(bar_tempty(acc));
-                    chunk(va, kc0);
+                uint32_t r[32];
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    tc::tmem_ld32(r, taddr + c * 32);
+                    tc::tmem_ld_wait(r);
+                    if (c == NCH - 1) {                                   // the last of this tile's accumulators are in registers
+                        tc::fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) tc::mbar_arrive(bar_tempty(acc));
+                    }
+                    chunk(r, kc0 + c * 32);
                 }
                 acc ^= 1;
             }
@@ -476,7 +510,8 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
 
     tc::fence_before_sync();
     __syncthreads();
-    if (warp == 2) {
+    if (warp == 0) {
+        __syncwarp();
         tc::fence_after_sync();
         tc::tmem_dealloc(tmem_base, 512);
     }
