@@ -263,47 +263,60 @@ __global__ void row_stats_kernel(const float* __restrict__ part_m, const float* 
 
 // Per unit: the mass every row puts on every shot, normalised and summed over the rows:
 //   unit_shot[u][i] = sum_r ( sum_{pieces q of shot i} z_q[r] * exp2(m_q[r] - m[r]) ) / Z[r]
-// One thread per row; pieces of one shot are consecutive in the piece list (piece_seg ascending,
-// segment 0 = tokens before the first shot, 1..S = shots, S+1 = the question).
+// One thread per row.  Each thread first reduces its row's pieces to (m, 1/Z), then walks the
+// pieces again and the rows of every piece are summed with warp shuffles into shared memory
+// (no block barrier per piece); a last pass adds the warps' partials and the pieces of each shot
+// in index order.  piece_seg is ascending: 0 = tokens before the first shot, 1..S = shots,
+// S+1 = the question, larger = list padding.  Shared memory: P * (THREADS/32 + 1) floats.
 template <int THREADS>
 __global__ void __launch_bounds__(THREADS) shot_mass_kernel(const float* __restrict__ part_m,
                                                            const float* __restrict__ part_z,
                                                            const int* __restrict__ piece_seg, int P, int R, int Rpad,
                                                            int L, int Hkv, int S, float* __restrict__ unit_shot) {
-    __shared__ float red[THREADS / 32];
+    constexpr int NW = THREADS / 32;
+    extern __shared__ float sm_mass[];          // [P][NW] warp partials, then [P] piece masses
+    float* piece_mass = sm_mass + (size_t)P * NW;
     const int u = blockIdx.x;
     const int b = u / (L * Hkv);
-    const int r = threadIdx.x;
+    const int r = threadIdx.x, warp = r >> 5, lane = r & 31;
     const int* seg = piece_seg + (size_t)b * P;
     const float* pm = part_m + (size_t)u * P * Rpad + r;
     const float* pz = part_z + (size_t)u * P * Rpad + r;
     const bool live = r < R;
+    int nreal = 0;                               // pieces that are not list padding (they come first)
+    while (nreal < P && seg[nreal] <= S + 1) ++nreal;
     float m = SHOTKV_NEG_INF, z = 0.f;
     if (live) {
-        for (int q = 0; q < P; ++q)
-            if (seg[q] <= S + 1) m = fmaxf(m, pm[(size_t)q * Rpad]);      // ids above S+1 are list padding
-        for (int q = 0; q < P; ++q)
-            if (seg[q] <= S + 1) z += pz[(size_t)q * Rpad] * ex2f(pm[(size_t)q * Rpad] - m);
+#pragma unroll 4
+        for (int q = 0; q < nreal; ++q) m = fmaxf(m, pm[(size_t)q * Rpad]);
+#pragma unroll 4
+        for (int q = 0; q < nreal; ++q) z += pz[(size_t)q * Rpad] * ex2f(pm[(size_t)q * Rpad] - m);
     }
     const float invz = (live && z > 0.f) ? 1.f / z : 0.f;
-    int q = 0;
-    while (q < P && seg[q] < 1) ++q;   // skip the pieces before the first shot
-    for (int i = 0; i < S; ++i) {
-        float a = 0.f;
-        while (q < P && seg[q] == i + 1) {
-            if (live) a += pz[(size_t)q * Rpad] * ex2f(pm[(size_t)q * Rpad] - m);
-            ++q;
-        }
-        a = warp_sum(a * invz);
-        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = a;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            float s = 0.f;
+#pragma unroll 4
+    for (int q = 0; q < nreal; ++q) {
+        float a = live ? pz[(size_t)q * Rpad] * ex2f(pm[(size_t)q * Rpad] - m) * invz : 0.f;
+        a = warp_sum(a);
+        if (lane == 0) sm_mass[q * NW + warp] = a;
+    }
+    __syncthreads();
+    for (int q = threadIdx.x; q < nreal; q += THREADS) {
+        float s = 0.f;
 #pragma unroll
-            for (int w = 0; w < THREADS / 32; ++w) s += red[w];
-            unit_shot[(size_t)u * S + i] = s;
+        for (int w = 0; w < NW; ++w) s += sm_mass[q * NW + w];
+        piece_mass[q] = s;
+    }
+    __syncthreads();
+    // shot i owns the consecutive pieces with seg == i + 1; find them by binary search
+    for (int i = threadIdx.x; i < S; i += THREADS) {
+        int lo = 0, hi = nreal;
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (seg[mid] < i + 1) lo = mid + 1; else hi = mid;
         }
-        __syncthreads();
+        float s = 0.f;
+        for (int q = lo; q < nreal && seg[q] == i + 1; ++q) s += piece_mass[q];
+        unit_shot[(size_t)u * S + i] = s;
     }
 }
 

@@ -98,6 +98,25 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// The same for the single-thread producer and MMA roles, which wait long and often: sleeping
+// between polls keeps their spinning out of the issue slots the epilogue warps need.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* err) {
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t spin = 1;; ++spin) {
+        __nanosleep(100);
+        if (mbar_try(bar, parity)) return true;
+        if ((spin & 15u) == 0u) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitCycles) {
+                *abort_flag = 1;
+                atomicExch(err, 1);
+                return false;
+            }
+        }
+    }
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                  ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
@@ -155,6 +174,20 @@ __device__ __forceinline__ void tmem_ld32(uint32_t (&v)[32], uint32_t taddr) {
         : "r"(taddr)
         : "memory");
 }
+// The same, and waits for the data: one statement, so the registers are defined when it ends.
+__device__ __forceinline__ void tmem_ld32_sync(uint32_t (&v)[32], uint32_t taddr) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
 // Waits for this thread's tensor-memory loads.  The registers are named as in/out operands so
 // that no use of them can be scheduled before the wait.
 __device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[32]) {
@@ -189,16 +222,42 @@ __device__ __forceinline__ void mask32(uint32_t (&r)[32], int valid) {
     for (int i = 0; i < 32; ++i)
         if (i >= valid) r[i] = 0xff800000u;
 }
-// sum of exp2(x*scale + neg)
+// Two fp32 values in one 64-bit register, for the packed fp32 instructions of sm_100.
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+    uint64_t v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(a), "f"(b));
+    return v;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// sum of exp2(x*scale + neg).  The multiply-add and the accumulation run two columns per
+// instruction: beside each exp2 on the special-function unit only about two and a half other
+// instructions can issue, so every instruction per column counts.
 __device__ __forceinline__ float expsum32(const uint32_t (&r)[32], float scale, float neg) {
-    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+    const uint64_t sc2 = pack2(scale, scale), ng2 = pack2(neg, neg);
+    uint64_t a0 = pack2(0.f, 0.f), a1 = a0;
 #pragma unroll
     for (int i = 0; i < 32; i += 4) {
-        s0 += ex2f(fmaf(SKV_F(r, i), scale, neg));
-        s1 += ex2f(fmaf(SKV_F(r, i + 1), scale, neg));
-        s2 += ex2f(fmaf(SKV_F(r, i + 2), scale, neg));
-        s3 += ex2f(fmaf(SKV_F(r, i + 3), scale, neg));
+        float x0, x1, x2, x3;
+        unpack2(ffma2(pack2(SKV_F(r, i), SKV_F(r, i + 1)), sc2, ng2), x0, x1);
+        unpack2(ffma2(pack2(SKV_F(r, i + 2), SKV_F(r, i + 3)), sc2, ng2), x2, x3);
+        a0 = fadd2(a0, pack2(ex2f(x0), ex2f(x1)));
+        a1 = fadd2(a1, pack2(ex2f(x2), ex2f(x3)));
     }
+    float s0, s1, s2, s3;
+    unpack2(a0, s0, s1);
+    unpack2(a1, s2, s3);
     return (s0 + s1) + (s2 + s3);
 }
 // exp2(x*scale + neg) in place
@@ -305,7 +364,7 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
                 const int nt = (hi - lo + TN - 1) / TN;
                 if (nt <= 0) continue;
                 if (u != cur_u) {
-                    if (!(ok = tc::mbar_wait(bar_qempty, qephase, abort_flag, p.err))) break;
+                    if (!(ok = tc::mbar_wait_relaxed(bar_qempty, qephase, abort_flag, p.err))) break;
                     qephase ^= 1;
                     tc::mbar_expect_tx(bar_qfull, MB * NSUB * q_box_rows * 128);
 #pragma unroll
@@ -316,7 +375,7 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
                     cur_u = u;
                 }
                 for (int t = 0; t < nt; ++t) {
-                    if (!(ok = tc::mbar_wait(bar_empty(stage), ephase, abort_flag, p.err))) break;
+                    if (!(ok = tc::mbar_wait_relaxed(bar_empty(stage), ephase, abort_flag, p.err))) break;
                     tc::mbar_expect_tx(bar_full(stage), NSUB * k_box_rows * 128);
 #pragma unroll
                     for (int sub = 0; sub < NSUB; ++sub)
@@ -358,14 +417,14 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
                 if (nt <= 0) continue;
                 if (u != cur_u) {
                     if (cur_u >= 0) tc::umma_commit(bar_qempty);     // Q may be replaced once these MMAs are done
-                    if (!(ok = tc::mbar_wait(bar_qfull, qfphase, abort_flag, p.err))) break;
+                    if (!(ok = tc::mbar_wait_relaxed(bar_qfull, qfphase, abort_flag, p.err))) break;
                     qfphase ^= 1;
                     cur_u = u;
                 }
                 for (int t = 0; t < nt; ++t) {
-                    if (!(ok = tc::mbar_wait(bar_full(stage), fphase, abort_flag, p.err))) break;
+                    if (!(ok = tc::mbar_wait_relaxed(bar_full(stage), fphase, abort_flag, p.err))) break;
                     const uint32_t tph = acc ? tephase1 : tephase0;
-                    if (!(ok = tc::mbar_wait(bar_tempty(acc), tph, abort_flag, p.err))) break;
+                    if (!(ok = tc::mbar_wait_relaxed(bar_tempty(acc), tph, abort_flag, p.err))) break;
                     if (acc) tephase1 ^= 1; else tephase0 ^= 1;
                     tc::fence_after_sync();
                     const uint32_t kb = sK + stage * Cfg::kStageBytes;
@@ -414,6 +473,7 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
             const int pi_last = p.chunk_first[(size_t)bprompt * p.cf_stride + j + 1];
             int pend = pi < pi_last ? pcs[pi].y : 0x7fffffff;
             float m_ref = SHOTKV_NEG_INF, z = 0.f;
+            const int plain_end = min(hi, p.N - p.W + 1);      // keys below this count for every window row
 
             // piece `pi` is complete for this thread's columns: merge the row's slices, write, move on
             auto flush = [&]() {
@@ -482,24 +542,36 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
 
             for (int t = 0; t < nt; ++t) {
                 const uint32_t tph = acc ? tfphase1 : tfphase0;
-                ok = tc::mbar_wait(bar_tfull(acc), tph, abort_flag, p.err);
-                ok = __all_sync(0xffffffffu, ok);
+                ok = lane == 0 ? tc::mbar_wait(bar_tfull(acc), tph, abort_flag, p.err) : true;   // one poller per warp
+                ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) break;
                 if (acc) tfphase1 ^= 1; else tfphase0 ^= 1;
                 tc::fence_after_sync();
                 const int kc0 = lo + t * TN + slice * SLW;
                 const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)((acc * MB + blk) * TN + slice * SLW);
+                while (pend <= kc0) flush();
+                // most tiles: every column of the slice counts for every row (it lies before the item's
+                // end and before the first window position) and no piece ends inside it
+                const bool plain = kc0 + SLW <= min(pend, plain_end);
                 uint32_t r[32];
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) {
-                    tc::tmem_ld32(r, taddr + c * 32);
-                    tc::tmem_ld_wait(r);
+                    tc::tmem_ld32_sync(r, taddr + c * 32);
                     if (c == NCH - 1) {                                   // the last of this tile's accumulators are in registers
                         tc::fence_before_sync();
                         __syncwarp();
                         if (lane == 0) tc::mbar_arrive(bar_tempty(acc));
                     }
-                    chunk(r, kc0 + c * 32);
+                    if (plain) {
+                        const float cm = tc::max32(r) * scale;
+                        if (cm > m_ref + 8.f) {
+                            z *= ex2f(m_ref - cm);
+                            m_ref = cm;
+                        }
+                        z += tc::expsum32(r, scale, -m_ref);
+                    } else {
+                        chunk(r, kc0 + c * 32);
+                    }
                 }
                 acc ^= 1;
             }

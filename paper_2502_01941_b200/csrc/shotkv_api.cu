@@ -696,10 +696,15 @@ int shotkv_prefill_compress(shotkv_ctx* ctx, const shotkv_dims* dims, const shot
     const int U = dims->B * dims->L * dims->Hkv;
     const int R = (dims->H / dims->Hkv) * dims->W, Rpad = rpad_of(dims);
     if (dims->S > 0) {
-        if (Rpad == 128)
-            shot_mass_kernel<128><<<U, 128, 0, stream>>>(w.part_m, w.part_z, w.piece_seg, P, R, Rpad, dims->L, dims->Hkv, dims->S, w.unit_shot);
-        else
-            shot_mass_kernel<256><<<U, 256, 0, stream>>>(w.part_m, w.part_z, w.piece_seg, P, R, Rpad, dims->L, dims->Hkv, dims->S, w.unit_shot);
+        const size_t msm = (size_t)P * (Rpad / 32 + 1) * 4;
+        if (msm > 200 * 1024) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "too many shots for the single-pass path (S = %d)", dims->S);
+        if (Rpad == 128) {
+            if (msm > 48 * 1024) CUDA_TRY(ctx, cudaFuncSetAttribute(shot_mass_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)msm));
+            shot_mass_kernel<128><<<U, 128, msm, stream>>>(w.part_m, w.part_z, w.piece_seg, P, R, Rpad, dims->L, dims->Hkv, dims->S, w.unit_shot);
+        } else {
+            if (msm > 48 * 1024) CUDA_TRY(ctx, cudaFuncSetAttribute(shot_mass_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)msm));
+            shot_mass_kernel<256><<<U, 256, msm, stream>>>(w.part_m, w.part_z, w.piece_seg, P, R, Rpad, dims->L, dims->Hkv, dims->S, w.unit_shot);
+        }
         LAUNCH_CHECK(ctx);
         shot_score_from_mass_kernel<<<dims->B * dims->L, 128, 0, stream>>>(w.unit_shot, w.off, dims->L, dims->Hkv, dims->S, shot_scores);
         LAUNCH_CHECK(ctx);
