@@ -316,9 +316,11 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
     auto bar_full = [&](int s) { return sBar + 8u * s; };
     auto bar_empty = [&](int s) { return sBar + 8u * (NST + s); };
     const uint32_t bar_qfull = sBar + 8u * (2 * NST), bar_qempty = bar_qfull + 8u;
-    auto bar_tfull = [&](int a) { return sBar + 8u * (2 * NST + 2 + a); };
-    auto bar_tempty = [&](int a) { return sBar + 8u * (2 * NST + 4 + a); };
-    const uint32_t tmem_slot = sBar + 8u * (2 * NST + 6);
+    // accumulator-ready / accumulator-free barriers per (buffer, row block): the two row blocks of a
+    // tile are handed over separately, which keeps their epilogue warps half a chunk out of phase
+    auto bar_tfull = [&](int a, int b) { return sBar + 8u * (2 * NST + 2 + a * 2 + b); };
+    auto bar_tempty = [&](int a, int b) { return sBar + 8u * (2 * NST + 6 + a * 2 + b); };
+    const uint32_t tmem_slot = sBar + 8u * (2 * NST + 10);
     volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(gbase + (tmem_slot - base));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + (tmem_slot - base) + 4);
     float* comb = reinterpret_cast<float*>(gbase + (sBar - base) + Cfg::kBarBytes);   // [2][4][128][2]
@@ -332,10 +334,11 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
         }
         tc::mbar_init(bar_qfull, 1);
         tc::mbar_init(bar_qempty, 1);
-        for (int a = 0; a < 2; ++a) {
-            tc::mbar_init(bar_tfull(a), 1);
-            tc::mbar_init(bar_tempty(a), 16);     // one arrival per epilogue warp
-        }
+        for (int a = 0; a < 2; ++a)
+            for (int b = 0; b < 2; ++b) {
+                tc::mbar_init(bar_tfull(a, b), 1);
+                tc::mbar_init(bar_tempty(a, b), 16 / MB);     // one arrival per epilogue warp of the row block
+            }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -424,12 +427,11 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
                 for (int t = 0; t < nt; ++t) {
                     if (!(ok = tc::mbar_wait_relaxed(bar_full(stage), fphase, abort_flag, p.err))) break;
                     const uint32_t tph = acc ? tephase1 : tephase0;
-                    if (!(ok = tc::mbar_wait_relaxed(bar_tempty(acc), tph, abort_flag, p.err))) break;
-                    if (acc) tephase1 ^= 1; else tephase0 ^= 1;
-                    tc::fence_after_sync();
                     const uint32_t kb = sK + stage * Cfg::kStageBytes;
 #pragma unroll
                     for (int b = 0; b < MB; ++b) {
+                        if (!(ok = tc::mbar_wait_relaxed(bar_tempty(acc, b), tph, abort_flag, p.err))) break;
+                        tc::fence_after_sync();
                         const uint32_t d_tmem = tmem_base + (uint32_t)((acc * MB + b) * TN);
 #pragma unroll
                         for (int ks = 0; ks < KSTEPS; ++ks) {
@@ -437,9 +439,11 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
                             const uint32_t b_addr = kb + (ks >> 2) * Cfg::kSubBytes + (ks & 3) * 32;
                             tc::umma_bf16(d_tmem, tc::smem_desc(a_addr), tc::smem_desc(b_addr), idesc, ks > 0);
                         }
+                        tc::umma_commit(bar_tfull(acc, b));
                     }
+                    if (!ok) break;
+                    if (acc) tephase1 ^= 1; else tephase0 ^= 1;
                     tc::umma_commit(bar_empty(stage));
-                    tc::umma_commit(bar_tfull(acc));
                     if (++stage == NST) {
                         stage = 0;
                         fphase ^= 1;
@@ -542,7 +546,7 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
 
             for (int t = 0; t < nt; ++t) {
                 const uint32_t tph = acc ? tfphase1 : tfphase0;
-                ok = lane == 0 ? tc::mbar_wait(bar_tfull(acc), tph, abort_flag, p.err) : true;   // one poller per warp
+                ok = lane == 0 ? tc::mbar_wait(bar_tfull(acc, blk), tph, abort_flag, p.err) : true;   // one poller per warp
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) break;
                 if (acc) tfphase1 ^= 1; else tfphase0 ^= 1;
@@ -560,7 +564,7 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
                     if (c == NCH - 1) {                                   // the last of this tile's accumulators are in registers
                         tc::fence_before_sync();
                         __syncwarp();
-                        if (lane == 0) tc::mbar_arrive(bar_tempty(acc));
+                        if (lane == 0) tc::mbar_arrive(bar_tempty(acc, blk));
                     }
                     if (plain) {
                         const float cm = tc::max32(r) * scale;
