@@ -41,6 +41,9 @@ from paper_2502_01941_b200 import workloads as wl
 METRIC = "prompt tokens compressed/sec"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
+# DRAM traffic of the scoring kernel per algorithmic K byte, from the ncu capture summarised in
+# profiles/score_tc_kernel_cfg3_B1_L8.md; set to None whenever the kernel changes after the capture.
+SCORE_TC_TRAFFIC_RATIO = 1.043
 NOMINAL_HBM_GBS = 8000.0
 
 
@@ -199,23 +202,34 @@ def run_ours(args):
     launches = skv.shotkv_launch_count(ctx) - launches0
     ms_total = max_over_ranks(e0.elapsed_time(e1), world, dev)
     ms_step = ms_total / args.steps
-    stages = np.array([skv.shotkv_profile_read(ctx, i) for i in range(min(args.steps, 64))])   # [calls][3]
+    stages = np.array([skv.shotkv_profile_read(ctx, i) for i in range(min(args.steps, 64))])   # [calls][4]
     skv.shotkv_profile_enable(ctx, False)
     kept = out["kept_count"].cpu().numpy()
     ab = algorithmic_bytes(cfg, kept)
-    score_ms, select_ms, compact_ms = [float(x) for x in stages.mean(axis=0)]
+    score_ms, reduce_ms, select_ms, compact_ms = [float(x) for x in stages.mean(axis=0)]
     tokens = cfg.B * cfg.N * world
     value = tokens / (ms_step * 1e-3)
     achieved = ab["k_read"] / (score_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "window scoring (QK^T + softmax partials), one launch per step",
+    logits = cfg.B * cfg.L * cfg.H * cfg.W * cfg.N                       # one ex2 per window logit
+    sm_mhz = clocks.get("sm_mhz") or 1965.0
+    ex2_rate = logits / (score_ms * 1e-3) / 148 / (sm_mhz * 1e6)
+    roofline = {"bound": "hbm", "kernel": "score_tc_kernel (window QK^T on tcgen05 + softmax partials), one launch per step",
                 "achieved": round(achieved, 1), "peak": peak, "peak_source": peak_src, "unit": "GB/s",
-                "frac": round(achieved / peak, 4), "traffic": None,
-                "algorithmic_bytes_per_launch": ab["k_read"], "ms_per_launch": round(score_ms, 4)}
+                "frac": round(achieved / peak, 4),
+                # dram__bytes_read+write of this kernel on the B=1, L=8 copy of the workload (profiles/
+                # score_tc_kernel_cfg3_B1_L8.md: 1.043 x its K bytes), scaled by the K bytes of a full launch
+                "traffic": int(SCORE_TC_TRAFFIC_RATIO * ab["k_read"]) if SCORE_TC_TRAFFIC_RATIO else None,
+                "algorithmic_bytes_per_launch": ab["k_read"], "ms_per_launch": round(score_ms, 4),
+                # what actually limits this kernel: one ex2 per logit on the special-function unit
+                # (16 lanes/clk/SM measured) and the issue slots around it
+                "also": {"bound": "alu", "unit": "ex2/clk/SM", "achieved": round(ex2_rate, 2), "peak": 16.0,
+                         "frac": round(ex2_rate / 16.0, 4), "at_sm_mhz": sm_mhz}}
     path = {"bytes_per_step": ab["total"], "k_read_bytes": ab["k_read"], "kv_gathered_bytes": ab["kv_gathered"],
             "achieved_gbs": round(ab["total"] / (ms_step * 1e-3) / 1e9, 1),
             "frac_of_measured_hbm": round(ab["total"] / (ms_step * 1e-3) / 1e9 / peak, 4),
             "frac_of_nominal_8tbs": round(ab["total"] / (ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS, 4),
-            "stage_ms": {"score": round(score_ms, 4), "select": round(select_ms, 4), "compact": round(compact_ms, 4)},
+            "stage_ms": {"score": round(score_ms, 4), "shot_reduce": round(reduce_ms, 4), "select": round(select_ms, 4),
+                         "compact": round(compact_ms, 4)},
             "compact_gbs": round(ab["kv_gathered"] / (compact_ms * 1e-3) / 1e9, 1),
             "kept_tokens_mean": float(kept.mean()), "budget_tokens": skv.shotkv_budget_tokens(dims, pol)}
 
@@ -287,9 +301,9 @@ def decode_leg(skv, ctx, rank, world, dev, peak, args) -> dict:
     """Config 4: batch 8 x 32 layers; the compressed prefill cache comes from running Phase 1 on a
     config-2-shaped batch of 8 prompts; then 1,024 decode steps, evicting to 25% every 32 steps."""
     dc = wl.DECODE_CONFIG
-    if args.decode_steps:
+    if args.decode_steps or args.decode_batch:
         import dataclasses
-        dc = dataclasses.replace(dc, steps=args.decode_steps)
+        dc = dataclasses.replace(dc, steps=args.decode_steps or dc.steps, B=args.decode_batch or dc.B)
     pc = rank_config(wl.CONFIGS[2].replace(B=dc.B), rank)
     dims = skv.make_dims(pc.B, pc.L, pc.H, pc.Hkv, pc.d, pc.N, pc.W, pc.S)
     pol = skv.make_policy(r_p=pc.r_p, r_d=dc.r_d, recompress_every=dc.recompress_every)
@@ -332,7 +346,7 @@ def decode_leg(skv, ctx, rank, world, dev, peak, args) -> dict:
     barrier(world)
     ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
     launches = skv.shotkv_launch_count(ctx) - l0
-    st_ms = np.array([skv.shotkv_profile_read(ctx, i)[:2] for i in range(64)])
+    st_ms = np.array([skv.shotkv_profile_read(ctx, i)[:2] for i in range(min(64, dc.steps))])
     skv.shotkv_profile_enable(ctx, False)
     per_step_bytes = bytes_read / dc.steps
     score_ms = float(st_ms[:, 0].mean())
@@ -420,6 +434,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override B (profiler captures of a smaller case)")
     ap.add_argument("--layers", type=int, default=0, help="override L (profiler captures of a smaller case)")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the number of decode steps")
+    ap.add_argument("--decode-batch", type=int, default=0, help="override the decode batch (profiler captures)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")

@@ -232,15 +232,26 @@ SHOTKV_API int shotkv_decode_step(shotkv_ctx* ctx, shotkv_decode_state* state,
                        const shotkv_bf16* q, const shotkv_bf16* k_new, const shotkv_bf16* v_new,
                        const shotkv_bf16* Kc, const int32_t* kept_count, void* stream);
 
+/* The work partition the scoring pass uses for `dims` on a GPU with `sm_count` SMs (host only; a
+ * diagnostic and test aid).  Every prompt's keys [0, N) are cut into pieces at the shot boundaries
+ * (when offsets_host is given) and at the ends of `nchunk` equal chunks of `chunk_keys` keys (whole
+ * 128-key tiles); per (piece, window row) the scoring kernel emits one softmax partial.
+ *   pieces_out  host [B][cap][3] = (lo, hi, segment) per piece; segment 0 = before the first shot,
+ *               i+1 = shot i, S+1 = the question, S+2 = list padding.  May be NULL.
+ * Returns the number of pieces per prompt (<= S + 67), or a negative error.  */
+SHOTKV_API int32_t shotkv_plan_pieces(const shotkv_dims* dims, const int32_t* offsets_host, int32_t sm_count,
+                           int32_t* nchunk, int32_t* chunk_keys, int32_t* pieces_out, int32_t cap);
+
 /* ---- instrumentation (used by the benchmark; not part of the method) ------------------------ */
 
 /* When enabled, shotkv_prefill_compress (single-pass form) and shotkv_decode_step record CUDA
  * events on their stream at their stage boundaries; the last 64 calls are retained.  */
 SHOTKV_API int shotkv_profile_enable(shotkv_ctx* ctx, int enable);
 /* Stage durations in milliseconds of the profiled call made `calls_back` calls ago (0 = latest);
- * waits for that call to finish.  Prefill: {score+per-shot reduce, select, compact};
- * decode: {score kernel, accumulate+evict, -1}.  Returns the number of stages or a negative error. */
-SHOTKV_API int shotkv_profile_read(shotkv_ctx* ctx, int calls_back, float* stage_ms /* [3] */);
+ * waits for that call to finish.  Prefill: {scoring kernel, per-shot reduce, select, compact};
+ * decode: {score kernel, accumulate+evict, -1, -1}.  Returns the number of stages or a negative
+ * error. */
+SHOTKV_API int shotkv_profile_read(shotkv_ctx* ctx, int calls_back, float* stage_ms /* [4] */);
 /* Kernels launched through this context since it was created. */
 SHOTKV_API uint64_t shotkv_launch_count(const shotkv_ctx* ctx);
 

@@ -32,7 +32,7 @@ EXPORTS = [
     "shotkv_prefill_score", "shotkv_select_shots", "shotkv_compact_kv", "shotkv_prefill_compress",
     "shotkv_host_arena_bytes", "shotkv_prefill_compress_host",
     "shotkv_decode_workspace_bytes", "shotkv_decode_capacity", "shotkv_decode_init", "shotkv_decode_step",
-    "shotkv_profile_enable", "shotkv_profile_read", "shotkv_launch_count", "shotkv_select_shots_static",
+    "shotkv_profile_enable", "shotkv_profile_read", "shotkv_launch_count", "shotkv_select_shots_static", "shotkv_plan_pieces",
 ]
 
 
@@ -92,6 +92,7 @@ def lib() -> C.CDLL:
         "shotkv_decode_capacity": (i32, [PP, i32]),
         "shotkv_decode_init": (C.c_int, [vp, PD, PP, i32, i32, vp, vp, vp, vp, vp, sz, C.POINTER(DecodeState)]),
         "shotkv_decode_step": (C.c_int, [vp, C.POINTER(DecodeState), vp, vp, vp, vp, vp, vp]),
+        "shotkv_plan_pieces": (i32, [PD, vp, i32, C.POINTER(i32), C.POINTER(i32), vp, i32]),
         "shotkv_profile_enable": (C.c_int, [vp, C.c_int]),
         "shotkv_profile_read": (C.c_int, [vp, C.c_int, C.POINTER(C.c_float)]),
         "shotkv_launch_count": (C.c_uint64, [vp]),
@@ -314,12 +315,25 @@ def shotkv_decode_step(ctx: Context, state: DecodeState, q, k_new, v_new, Kc, ke
     return ctx.check(rc)
 
 
+def shotkv_plan_pieces(dims: Dims, offsets=None, sm_count: int = 148):
+    """(nchunk, chunk_keys, pieces [B][P][3]) of the scoring pass's work partition (host only)."""
+    o = _offsets(offsets) if offsets is not None else None
+    cap = dims.S + 80
+    out = np.zeros((dims.B, cap, 3), dtype=np.int32)
+    nchunk, ck = C.c_int32(), C.c_int32()
+    P = int(lib().shotkv_plan_pieces(C.byref(dims), o.ctypes.data_as(C.c_void_p) if o is not None else None, int(sm_count),
+                                     C.byref(nchunk), C.byref(ck), out.ctypes.data_as(C.c_void_p), cap))
+    if P < 0:
+        raise ShotKVError(P, "shotkv_plan_pieces rejected its arguments")
+    return int(nchunk.value), int(ck.value), out[:, :P, :].copy()
+
+
 def shotkv_profile_enable(ctx: Context, enable: bool) -> int:
     return ctx.check(lib().shotkv_profile_enable(ctx._h, int(bool(enable))))
 
 
 def shotkv_profile_read(ctx: Context, calls_back: int = 0) -> list:
-    ms = (C.c_float * 3)()
+    ms = (C.c_float * 4)()
     n = ctx.check(lib().shotkv_profile_read(ctx._h, int(calls_back), ms))
     return [float(ms[i]) for i in range(n)]
 

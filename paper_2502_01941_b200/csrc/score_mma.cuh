@@ -1,15 +1,14 @@
-// Window attention scoring with warp-level MMA (mma.sync m16n8k16, bf16 in, fp32 accumulate).
+// Second pass of per-token importance, and the small reductions that follow the scoring pass.
 //
-// One CTA owns one (prompt, layer, kv head) unit's R = G*W window rows (padded to 128 or 256)
-// and walks a list of key ranges ("pieces").  Q stays in registers as A fragments; K tiles of 64
-// keys are staged in shared memory with cp.async (double buffered) and read with ldmatrix.
+// column_sum_mma_kernel: with every window row's final maximum and 1/Z known (row_stats_kernel),
+// the logits are recomputed with warp-level MMA (mma.sync m16n8k16, bf16 in, fp32 accumulate),
+// normalised and summed over the rows: token_importance[t] = sum_r alpha[r][t].  One CTA owns a
+// unit's R = G*W window rows (padded to 128 or 256, Q held in registers as A fragments) and walks
+// a list of key ranges; K tiles of 64 keys are staged in shared memory with cp.async (double
+// buffered) and read with ldmatrix.
 //
-//   STATS  : per piece and row, the maximum logit m and z = sum exp2(x - m) over the piece
-//            (x = q.k * log2(e)/sqrt(d)).  Pieces never straddle a shot boundary, so the same
-//            partials give both the softmax denominator of every row and, per shot, the mass
-//            the row puts on that shot.
-//   COLSUM : with the final row maxima and 1/Z known, the normalised weights are recomputed
-//            and summed over the rows: token_importance[t] = sum_r alpha[r][t].
+// row_stats_kernel, shot_mass_kernel, shot_score_from_mass_kernel: fixed-order reductions of the
+// per-(piece, row) partials (m, z) written by the tensor-core scoring kernel.
 #pragma once
 #include "common.cuh"
 
@@ -22,11 +21,9 @@ struct ScoreParams {
     int P, ppc;               // pieces per prompt, pieces per CTA
     int L, H, Hkv, N, W, G, R, Rpad;
     float scale_log2;         // log2(e)/sqrt(d)
-    float* part_m;            // [U][P][Rpad]   STATS out
-    float* part_z;            // [U][P][Rpad]   STATS out
-    const float* row_m;       // [U][Rpad]      COLSUM in
-    const float* row_invz;    // [U][Rpad]      COLSUM in (0 for padding rows)
-    float* imp;               // [U][N]         COLSUM out
+    const float* row_m;       // [U][Rpad]      final row maxima (log2 domain)
+    const float* row_invz;    // [U][Rpad]      1/Z per row (0 for padding rows)
+    float* imp;               // [U][N]         out
 };
 
 constexpr int kTileKeys = 64;
@@ -36,8 +33,8 @@ constexpr int score_mma_smem_bytes() {
     return 128 * MB * D * 2 + 2 * kTileKeys * D * 2 + 8 * kTileKeys * 4;
 }
 
-template <int D, int MB, bool COLSUM>
-__global__ void __launch_bounds__(256, (MB == 1 ? 2 : 1)) score_mma_kernel(const ScoreParams p) {
+template <int D, int MB>
+__global__ void __launch_bounds__(256, (MB == 1 ? 2 : 1)) column_sum_mma_kernel(const ScoreParams p) {
     constexpr int ROWB = D * 2;
     constexpr int CH = D / 8;
     constexpr int KS = D / 16;
@@ -85,13 +82,8 @@ __global__ void __launch_bounds__(256, (MB == 1 ? 2 : 1)) score_mma_kernel(const
         for (int hf = 0; hf < 2; ++hf) {
             const int r = mb * 128 + warp * 16 + g + hf * 8;
             plim[mb][hf] = r < p.R ? p.N - p.W + (r % p.W) : p.N - 1;
-            if (COLSUM) {
-                rm[mb][hf] = p.row_m[(size_t)u * p.Rpad + r];
-                rinv[mb][hf] = p.row_invz[(size_t)u * p.Rpad + r];
-            } else {
-                rm[mb][hf] = 0.f;
-                rinv[mb][hf] = 0.f;
-            }
+            rm[mb][hf] = p.row_m[(size_t)u * p.Rpad + r];
+            rinv[mb][hf] = p.row_invz[(size_t)u * p.Rpad + r];
         }
 
     const int piece_begin = blockIdx.x * p.ppc;
@@ -100,13 +92,6 @@ __global__ void __launch_bounds__(256, (MB == 1 ? 2 : 1)) score_mma_kernel(const
         const int2 pc = p.pieces[(size_t)b * p.P + pi];
         const int lo = pc.x, hi = pc.y;
         const int ntile = (hi - lo + TK - 1) / TK;
-        float m_run[MB][2], z_run[MB][2];
-#pragma unroll
-        for (int mb = 0; mb < MB; ++mb) {
-            m_run[mb][0] = m_run[mb][1] = SHOTKV_NEG_INF;
-            z_run[mb][0] = z_run[mb][1] = 0.f;
-        }
-
         auto load_tile = [&](int t) {
             const uint32_t dst = smem_u32(sK) + (t & 1) * TK * ROWB;
             const int key0 = lo + t * TK;
@@ -165,29 +150,7 @@ __global__ void __launch_bounds__(256, (MB == 1 ? 2 : 1)) score_mma_kernel(const
                         acc[mb][n][e] = ok ? acc[mb][n][e] * p.scale_log2 : SHOTKV_NEG_INF;
                     }
 
-            if (!COLSUM) {
-#pragma unroll
-                for (int mb = 0; mb < MB; ++mb)
-#pragma unroll
-                    for (int hf = 0; hf < 2; ++hf) {
-                        float tm = SHOTKV_NEG_INF;
-#pragma unroll
-                        for (int n = 0; n < 8; ++n) tm = fmaxf(tm, fmaxf(acc[mb][n][2 * hf], acc[mb][n][2 * hf + 1]));
-                        tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, 1));
-                        tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, 2));
-                        const float m_new = fmaxf(m_run[mb][hf], tm);
-                        // all-masked so far: keep z = 0 and avoid (-inf) - (-inf)
-                        const float m_use = m_new == SHOTKV_NEG_INF ? 0.f : m_new;
-                        float s = 0.f;
-#pragma unroll
-                        for (int n = 0; n < 8; ++n)
-                            s += ex2f(acc[mb][n][2 * hf] - m_use) + ex2f(acc[mb][n][2 * hf + 1] - m_use);
-                        s += __shfl_xor_sync(0xffffffffu, s, 1);
-                        s += __shfl_xor_sync(0xffffffffu, s, 2);
-                        z_run[mb][hf] = z_run[mb][hf] * ex2f(m_run[mb][hf] - m_use) + s;
-                        m_run[mb][hf] = m_new;
-                    }
-            } else {
+            {
 #pragma unroll
                 for (int n = 0; n < 8; ++n) {
                     float v0 = 0.f, v1 = 0.f;
@@ -218,18 +181,6 @@ __global__ void __launch_bounds__(256, (MB == 1 ? 2 : 1)) score_mma_kernel(const
                 }
             }
             __syncthreads();
-        }
-
-        if (!COLSUM && t4 == 0) {
-#pragma unroll
-            for (int mb = 0; mb < MB; ++mb)
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    const int r = mb * 128 + warp * 16 + g + hf * 8;
-                    const size_t o = ((size_t)u * p.P + pi) * p.Rpad + r;
-                    p.part_m[o] = m_run[mb][hf];
-                    p.part_z[o] = z_run[mb][hf];
-                }
         }
     }
 }
@@ -285,15 +236,20 @@ __global__ void __launch_bounds__(THREADS) shot_mass_kernel(const float* __restr
     const bool live = r < R;
     int nreal = 0;                               // pieces that are not list padding (they come first)
     while (nreal < P && seg[nreal] <= S + 1) ++nreal;
+    // one pass for (m, Z) with a running maximum, one pass for the masses
     float m = SHOTKV_NEG_INF, z = 0.f;
     if (live) {
-#pragma unroll 4
-        for (int q = 0; q < nreal; ++q) m = fmaxf(m, pm[(size_t)q * Rpad]);
-#pragma unroll 4
-        for (int q = 0; q < nreal; ++q) z += pz[(size_t)q * Rpad] * ex2f(pm[(size_t)q * Rpad] - m);
+#pragma unroll 8
+        for (int q = 0; q < nreal; ++q) {
+            const float mq = pm[(size_t)q * Rpad], zq = pz[(size_t)q * Rpad];
+            const float mn = fmaxf(m, mq);
+            const float mu = mn == SHOTKV_NEG_INF ? 0.f : mn;
+            z = z * ex2f(m - mu) + zq * ex2f(mq - mu);
+            m = mn;
+        }
     }
     const float invz = (live && z > 0.f) ? 1.f / z : 0.f;
-#pragma unroll 4
+#pragma unroll 8
     for (int q = 0; q < nreal; ++q) {
         float a = live ? pz[(size_t)q * Rpad] * ex2f(pm[(size_t)q * Rpad] - m) * invz : 0.f;
         a = warp_sum(a);

@@ -41,7 +41,7 @@ struct shotkv_ctx {
     int stage_next = 0;
     // optional stage timing: a ring of event sets, one per profiled call
     bool prof = false;
-    cudaEvent_t prof_ev[kProfSlots][4] = {};
+    cudaEvent_t prof_ev[kProfSlots][5] = {};
     int prof_marks[kProfSlots] = {};
     int prof_calls = 0;
     unsigned long long launches = 0;   // kernels launched through this context
@@ -87,7 +87,7 @@ void prof_mark(shotkv_ctx* ctx, cudaStream_t stream) {
     if (!ctx->prof || ctx->prof_calls == 0) return;
     const int slot = (ctx->prof_calls - 1) % kProfSlots;
     int& m = ctx->prof_marks[slot];
-    if (m < 4) cudaEventRecord(ctx->prof_ev[slot][m++], stream);
+    if (m < 5) cudaEventRecord(ctx->prof_ev[slot][m++], stream);
 }
 
 int check_dims(const shotkv_dims* d, const char** why) {
@@ -259,28 +259,20 @@ int build_pieces(const shotkv_dims* d, const int32_t* off, const ChunkPlan& plan
     return (int)P;
 }
 
-template <int D, int MB, bool COLSUM>
-int launch_score_t(shotkv_ctx* ctx, const ScoreParams& sp, int U, cudaStream_t stream) {
+template <int D, int MB>
+int launch_colsum_t(shotkv_ctx* ctx, const ScoreParams& sp, int U, cudaStream_t stream) {
     constexpr int smem = score_mma_smem_bytes<D, MB>();
-    static bool attr_done[64] = {};
-    int dev = ctx->device;
-    if (dev < 64 && !attr_done[dev]) {
-        CUDA_TRY(ctx, cudaFuncSetAttribute(score_mma_kernel<D, MB, COLSUM>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        attr_done[dev] = true;
-    } else if (dev >= 64) {
-        CUDA_TRY(ctx, cudaFuncSetAttribute(score_mma_kernel<D, MB, COLSUM>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    }
+    CUDA_TRY(ctx, cudaFuncSetAttribute(column_sum_mma_kernel<D, MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     dim3 grid((sp.P + sp.ppc - 1) / sp.ppc, U);
-    score_mma_kernel<D, MB, COLSUM><<<grid, 256, smem, stream>>>(sp);
+    column_sum_mma_kernel<D, MB><<<grid, 256, smem, stream>>>(sp);
     LAUNCH_CHECK(ctx);
     return SHOTKV_OK;
 }
 
-template <bool COLSUM>
-int launch_score(shotkv_ctx* ctx, const shotkv_dims* d, const ScoreParams& sp, int U, cudaStream_t stream) {
+int launch_colsum(shotkv_ctx* ctx, const shotkv_dims* d, const ScoreParams& sp, int U, cudaStream_t stream) {
     const bool big = sp.Rpad == 256;
-    if (d->d == 128) return big ? launch_score_t<128, 2, COLSUM>(ctx, sp, U, stream) : launch_score_t<128, 1, COLSUM>(ctx, sp, U, stream);
-    return big ? launch_score_t<64, 2, COLSUM>(ctx, sp, U, stream) : launch_score_t<64, 1, COLSUM>(ctx, sp, U, stream);
+    if (d->d == 128) return big ? launch_colsum_t<128, 2>(ctx, sp, U, stream) : launch_colsum_t<128, 1>(ctx, sp, U, stream);
+    return big ? launch_colsum_t<64, 2>(ctx, sp, U, stream) : launch_colsum_t<64, 1>(ctx, sp, U, stream);
 }
 
 ScoreParams base_params(const shotkv_dims* d, const shotkv_bf16* Q, const shotkv_bf16* K, const PrefillWs& w, int P) {
@@ -295,7 +287,6 @@ ScoreParams base_params(const shotkv_dims* d, const shotkv_bf16* Q, const shotkv
     sp.L = d->L; sp.H = d->H; sp.Hkv = d->Hkv; sp.N = d->N; sp.W = d->W;
     sp.G = d->H / d->Hkv; sp.R = sp.G * d->W; sp.Rpad = rpad_of(d);
     sp.scale_log2 = kLog2e / sqrtf((float)d->d);
-    sp.part_m = w.part_m; sp.part_z = w.part_z;
     sp.row_m = w.row_m; sp.row_invz = w.row_invz;
     sp.imp = nullptr;
     return sp;
@@ -410,9 +401,9 @@ int run_stats(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const
     const int U = d->B * d->L * d->Hkv;
     ScoreParams sp = base_params(d, Q, K, w, P);
     prof_mark(ctx, stream);
-    static const bool use_mma = getenv("SHOTKV_SCORE_MMA") != nullptr;      // development A/B switch
-    rc = use_mma ? launch_score<false>(ctx, d, sp, U, stream) : launch_score_tc(ctx, d, Q, K, w, P, plan, stream);
+    rc = launch_score_tc(ctx, d, Q, K, w, P, plan, stream);
     if (rc) return rc;
+    prof_mark(ctx, stream);
     if (need_rows) {
         row_stats_kernel<<<U, 256, 0, stream>>>(w.part_m, w.part_z, w.piece_seg, d->L * d->Hkv, d->S + 1, P, sp.R, sp.Rpad,
                                                 w.row_m, w.row_invz);
@@ -502,7 +493,7 @@ void shotkv_destroy(shotkv_ctx* ctx) {
     if (ctx->stage) cudaFreeHost(ctx->stage);
     if (ctx->err_host) cudaFreeHost(ctx->err_host);
     for (int i = 0; i < kProfSlots; ++i)
-        for (int j = 0; j < 4; ++j)
+        for (int j = 0; j < 5; ++j)
             if (ctx->prof_ev[i][j]) cudaEventDestroy(ctx->prof_ev[i][j]);
     delete ctx;
 }
@@ -560,7 +551,7 @@ int shotkv_prefill_score(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_
     if ((rc = run_stats(ctx, dims, Qwin, K, w, nullptr, true, &P, stream))) return rc;
     ScoreParams sp = base_params(dims, Qwin, K, w, P);
     sp.imp = token_importance;
-    return launch_score<true>(ctx, dims, sp, dims->B * dims->L * dims->Hkv, stream);
+    return launch_colsum(ctx, dims, sp, dims->B * dims->L * dims->Hkv, stream);
 }
 
 int shotkv_select_shots(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_policy* policy,
@@ -896,13 +887,39 @@ int shotkv_decode_step(shotkv_ctx* ctx, shotkv_decode_state* st, const shotkv_bf
     return SHOTKV_OK;
 }
 
+int32_t shotkv_plan_pieces(const shotkv_dims* dims, const int32_t* offsets_host, int32_t sm_count, int32_t* nchunk,
+                           int32_t* chunk_keys, int32_t* pieces_out, int32_t cap) {
+    const char* why = "";
+    int rc = check_dims(dims, &why);
+    if (rc) return rc;
+    if (offsets_host && (rc = check_offsets(dims, nullptr, offsets_host, nullptr, &why)) < 0) return rc;
+    if (sm_count < 1) return SHOTKV_ERR_INVALID_ARG;
+    const ChunkPlan plan = plan_chunks(dims, sm_count);
+    std::vector<int2> pieces;
+    std::vector<int> seg, chunk_first;
+    const int P = build_pieces(dims, offsets_host, plan, pieces, seg, chunk_first);
+    if (nchunk) *nchunk = plan.nchunk;
+    if (chunk_keys) *chunk_keys = plan.chunk_keys;
+    if (pieces_out) {
+        if (cap < P) return SHOTKV_ERR_INVALID_ARG;
+        for (int b = 0; b < dims->B; ++b)
+            for (int i = 0; i < P; ++i) {
+                int32_t* o = pieces_out + ((size_t)b * cap + i) * 3;
+                o[0] = pieces[(size_t)b * P + i].x;
+                o[1] = pieces[(size_t)b * P + i].y;
+                o[2] = seg[(size_t)b * P + i];
+            }
+    }
+    return P;
+}
+
 // ---- instrumentation ------------------------------------------------------------------------
 int shotkv_profile_enable(shotkv_ctx* ctx, int enable) {
     int rc = set_device(ctx);
     if (rc) return rc;
     if (enable && !ctx->prof_ev[0][0]) {
         for (int i = 0; i < kProfSlots; ++i)
-            for (int j = 0; j < 4; ++j) CUDA_TRY(ctx, cudaEventCreate(&ctx->prof_ev[i][j]));
+            for (int j = 0; j < 5; ++j) CUDA_TRY(ctx, cudaEventCreate(&ctx->prof_ev[i][j]));
     }
     ctx->prof = enable != 0;
     ctx->prof_calls = 0;
@@ -916,7 +933,7 @@ int shotkv_profile_read(shotkv_ctx* ctx, int calls_back, float* stage_ms) {
         return fail(ctx, SHOTKV_ERR_INVALID_ARG, "no profiled call %d calls back", calls_back);
     const int slot = (ctx->prof_calls - 1 - calls_back) % kProfSlots;
     const int m = ctx->prof_marks[slot];
-    for (int i = 0; i < 3; ++i) stage_ms[i] = -1.f;
+    for (int i = 0; i < 4; ++i) stage_ms[i] = -1.f;
     if (m < 2) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "that call recorded no stages");
     CUDA_TRY(ctx, cudaEventSynchronize(ctx->prof_ev[slot][m - 1]));
     for (int i = 0; i + 1 < m; ++i) CUDA_TRY(ctx, cudaEventElapsedTime(&stage_ms[i], ctx->prof_ev[slot][i], ctx->prof_ev[slot][i + 1]));

@@ -110,3 +110,30 @@ def test_workload_generator_shapes_and_determinism():
     q2, k2, v2 = wl.prefill_unit(cfg, 0, 0, wl.shot_offsets(cfg, 0))
     assert (wl.bf16_bits(k1) == wl.bf16_bits(k2)).all() and (wl.bf16_bits(q1) == wl.bf16_bits(q2)).all()
     assert k1.shape == (cfg.Hkv, cfg.N, cfg.d) and q1.shape == (cfg.H, cfg.W, cfg.d) and v1.shape == k1.shape
+
+
+@pytest.mark.parametrize("cid", [0, 1, 2, 3])
+def test_scoring_work_partition_covers_every_key_once(cid):
+    """Host logic of the scoring pass: pieces tile [0, N) exactly, never straddle a shot boundary or a
+    chunk end, carry the right segment ids in ascending order, and chunks are whole 128-key tiles."""
+    cfg = wl.CONFIGS[cid]
+    d = skv.make_dims(cfg.B, cfg.L, cfg.H, cfg.Hkv, cfg.d, cfg.N, cfg.W, cfg.S)
+    off = wl.all_shot_offsets(cfg)
+    for sm in (1, 148):
+        nchunk, ck, pieces = skv.shotkv_plan_pieces(d, off, sm)
+        assert ck % 128 == 0 and nchunk >= 1 and (nchunk - 1) * ck < cfg.N <= nchunk * ck
+        assert pieces.shape[1] <= cfg.S + 2 + 64 + 1
+        for b in range(cfg.B):
+            real = pieces[b][pieces[b][:, 2] <= cfg.S + 1]
+            assert real[0, 0] == 0 and real[-1, 1] == cfg.N
+            assert np.all(real[1:, 0] == real[:-1, 1]) and np.all(real[:, 1] > real[:, 0])
+            assert np.all(np.diff(real[:, 2]) >= 0)
+            bounds = np.concatenate([[0], off[b], [cfg.N]])
+            for lo, hi, seg in real:
+                assert bounds[seg] <= lo and hi <= bounds[seg + 1]           # inside its segment
+                assert lo // ck == (hi - 1) // ck                            # inside one chunk
+            pad = pieces[b][pieces[b][:, 2] > cfg.S + 1]
+            assert np.all(pad[:, 0] == pad[:, 1])
+    # without offsets: plain chunks
+    nchunk, ck, pieces = skv.shotkv_plan_pieces(d, None, 148)
+    assert pieces.shape[1] == nchunk and pieces[0, 0, 0] == 0 and pieces[0, -1, 1] == cfg.N
