@@ -44,6 +44,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the scoring kernel per algorithmic K byte, from the ncu capture summarised in
 # profiles/score_tc_kernel_cfg3_B1_L8.md; set to None whenever the kernel changes after the capture.
 SCORE_TC_TRAFFIC_RATIO = 1.043
+DECODE_TRAFFIC_RATIO = 1.012    # profiles/decode_score_kernel_cfg4_B2.md
 NOMINAL_HBM_GBS = 8000.0
 
 
@@ -358,7 +359,9 @@ def decode_leg(skv, ctx, rank, world, dev, peak, args) -> dict:
                        "Dcap": Dcap},
             "roofline": {"bound": "hbm", "kernel": "decode score kernel (last 64 steps)",
                          "achieved": round(per_step_bytes / (score_ms * 1e-3) / 1e9, 1), "peak": peak, "unit": "GB/s",
-                         "frac": round(per_step_bytes / (score_ms * 1e-3) / 1e9 / peak, 4), "traffic": None,
+                         "frac": round(per_step_bytes / (score_ms * 1e-3) / 1e9 / peak, 4),
+                         # profiles/decode_score_kernel_cfg4_B2.md: dram read+write = 1.012 x algorithmic
+                         "traffic": int(DECODE_TRAFFIC_RATIO * per_step_bytes) if DECODE_TRAFFIC_RATIO else None,
                          "algorithmic_bytes_per_launch": int(per_step_bytes), "ms_per_launch": round(score_ms, 4)},
             "path_frac_of_measured_hbm": round(per_step_bytes / (ms / dc.steps * 1e-3) / 1e9 / peak, 4)}
 

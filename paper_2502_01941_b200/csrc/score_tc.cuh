@@ -554,9 +554,6 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
                 const int kc0 = lo + t * TN + slice * SLW;
                 const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)((acc * MB + blk) * TN + slice * SLW);
                 while (pend <= kc0) flush();
-                // most tiles: every column of the slice counts for every row (it lies before the item's
-                // end and before the first window position) and no piece ends inside it
-                const bool plain = kc0 + SLW <= min(pend, plain_end);
                 uint32_t r[32];
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) {
@@ -566,7 +563,9 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
                         __syncwarp();
                         if (lane == 0) tc::mbar_arrive(bar_tempty(acc, blk));
                     }
-                    if (plain) {
+                    // most chunks: every column counts for every row (it lies before the item's end and
+                    // before the first window position) and no piece ends at or inside the chunk
+                    if (kc0 + c * 32 + 32 <= min(pend, plain_end)) {
                         const float cm = tc::max32(r) * scale;
                         if (cm > m_ref + 8.f) {
                             z *= ex2f(m_ref - cm);
