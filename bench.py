@@ -167,6 +167,7 @@ def run_ours(args):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     ctx = skv.Context(local)
+    skv.shotkv_set_scoring_mode(ctx, skv.SCORING_EXACT if args.scoring == "exact" else skv.SCORING_FAST)
     peak, peak_src = measured_peaks()
 
     cfg = rank_config(wl.CONFIGS[args.workload], rank)
@@ -438,6 +439,8 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override L (profiler captures of a smaller case)")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the number of decode steps")
     ap.add_argument("--decode-batch", type=int, default=0, help="override the decode batch (profiler captures)")
+    ap.add_argument("--scoring", default="fast", choices=["fast", "exact"],
+                    help="scoring kernel: the default pair (fast kernel + exact repair) or the exact kernel alone")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")

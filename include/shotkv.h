@@ -244,6 +244,22 @@ SHOTKV_API int32_t shotkv_plan_pieces(const shotkv_dims* dims, const int32_t* of
 
 /* ---- instrumentation (used by the benchmark; not part of the method) ------------------------ */
 
+/* How the window logits are exponentiated in the scoring pass (the alpha of the prefill score
+ * equation, Section 5.1).  Both modes compute the same softmax sums; they differ in how the
+ * reference exponent of a window row is chosen.
+ *   SHOTKV_SCORING_FAST (default): per work item the reference is fixed from the item's first
+ *     128 keys and sums are carried in fp32 with about 2^158 of headroom above it; any item
+ *     whose sums leave that range is recomputed on the device by the exact kernel, in the same
+ *     call, so the outputs are those of the exact mode up to fp32 rounding.
+ *   SHOTKV_SCORING_EXACT: every item runs the exact kernel (a running maximum per row).
+ * Takes effect for the calls that follow on this context.  */
+#define SHOTKV_SCORING_FAST 0
+#define SHOTKV_SCORING_EXACT 1
+SHOTKV_API int shotkv_set_scoring_mode(shotkv_ctx* ctx, int mode);
+/* Work items (a run of a unit's keys) that the exact kernel recomputed after the fast one, summed
+ * over the calls finished so far on this context.  A diagnostic: 0 on ordinary inputs.  */
+SHOTKV_API uint64_t shotkv_repaired_items(const shotkv_ctx* ctx);
+
 /* When enabled, shotkv_prefill_compress (single-pass form) and shotkv_decode_step record CUDA
  * events on their stream at their stage boundaries; the last 64 calls are retained.  */
 SHOTKV_API int shotkv_profile_enable(shotkv_ctx* ctx, int enable);

@@ -33,6 +33,7 @@ EXPORTS = [
     "shotkv_host_arena_bytes", "shotkv_prefill_compress_host",
     "shotkv_decode_workspace_bytes", "shotkv_decode_capacity", "shotkv_decode_init", "shotkv_decode_step",
     "shotkv_profile_enable", "shotkv_profile_read", "shotkv_launch_count", "shotkv_select_shots_static", "shotkv_plan_pieces",
+    "shotkv_set_scoring_mode", "shotkv_repaired_items",
 ]
 
 
@@ -96,6 +97,8 @@ def lib() -> C.CDLL:
         "shotkv_profile_enable": (C.c_int, [vp, C.c_int]),
         "shotkv_profile_read": (C.c_int, [vp, C.c_int, C.POINTER(C.c_float)]),
         "shotkv_launch_count": (C.c_uint64, [vp]),
+        "shotkv_set_scoring_mode": (C.c_int, [vp, C.c_int]),
+        "shotkv_repaired_items": (C.c_uint64, [vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(L, name)
@@ -328,6 +331,17 @@ def shotkv_plan_pieces(dims: Dims, offsets=None, sm_count: int = 148):
     return int(nchunk.value), int(ck.value), out[:, :P, :].copy()
 
 
+SCORING_FAST, SCORING_EXACT = 0, 1
+
+
+def shotkv_set_scoring_mode(ctx: Context, mode: int) -> int:
+    return ctx.check(lib().shotkv_set_scoring_mode(ctx._h, int(mode)))
+
+
+def shotkv_repaired_items(ctx: Context) -> int:
+    return int(lib().shotkv_repaired_items(ctx._h))
+
+
 def shotkv_profile_enable(ctx: Context, enable: bool) -> int:
     return ctx.check(lib().shotkv_profile_enable(ctx._h, int(bool(enable))))
 
@@ -362,4 +376,5 @@ __all__ = [n for n in dir() if n.startswith("shotkv_")] + [
     "Context", "Dims", "Policy", "DecodeState", "ShotKVError", "make_dims", "make_policy", "alloc_prefill_outputs",
     "OK", "ERR_INVALID_ARG", "ERR_UNSUPPORTED_SHAPE", "ERR_BAD_OFFSETS", "ERR_WORKSPACE_TOO_SMALL", "ERR_CUDA",
     "ERR_TIMEOUT", "WARN_BUDGET_BELOW_ALWAYS_KEPT", "FLAG_TOKEN_IMPORTANCE", "EXPORTS", "LIB_PATH", "lib",
+    "SCORING_FAST", "SCORING_EXACT", "shotkv_set_scoring_mode", "shotkv_repaired_items",
 ]

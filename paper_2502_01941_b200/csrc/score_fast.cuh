@@ -1,0 +1,309 @@
+// Window attention scoring, the kernel the prefill path runs first: the same TMA producer, MMA
+// issuer, work items and per-(piece, window row) outputs (m, z) as score_tc.cuh, with an epilogue
+// arranged for throughput.
+//
+//   * Sixteen epilogue warps, every thread one window row and one column slice of a tile (64 of
+//     128 columns with two row blocks, 32 with one), as in the exact kernel.  When a piece is
+//     complete the warps of the later slices hand their (m, z) to the warp of slice 0 through a
+//     small ring of shared-memory slots guarded by mbarriers, so no warp waits for another at a
+//     piece end unless it is a whole ring ahead of it.  The code of the inner loop is
+//     kept small (one copy of the chunk arithmetic, one of the boundary handling): the warps of
+//     three roles share the instruction cache.
+//   * No running maximum.  The reference exponent m of a (row, work item) is fixed from the
+//     item's first tile: that tile's row maximum lands on 2^-32, and every later logit of the
+//     item is exponentiated against the same m.  fp32 leaves about 2^+158 above that point and
+//     2^-94 below it; what underflows is below 2^-94 of a term the row's own softmax denominator
+//     contains, so it cannot matter to any score.  What overflows is caught: a partial sum that
+//     is not below 1e30 marks its item in `redo`, and a second launch (the exact kernel of
+//     score_tc.cuh with the same flags) recomputes marked items with a true running maximum.
+//   * One ex2 per logit is the ceiling of the special-function unit (16 lanes per clock per SM),
+//     so PE of every 16 column pairs take their exponentials on the FMA pipe instead: round to nearest
+//     integer n by the magic-number addition, a cubic in the remainder f in [-1/2, 1/2]
+//     (relative error below 7.5e-5), and n added into the exponent field.  The argument is
+//     clamped to [-125, 128] first, so the result is a normal number, or +inf at the top.
+#pragma once
+#include "score_tc.cuh"
+
+namespace shotkv {
+
+template <int D, int MB>
+struct ScoreFastCfg {
+    static constexpr int kSub = D / 64;
+    static constexpr int kSubBytes = 128 * 128;
+    static constexpr int kQBytes = MB * kSub * kSubBytes;
+    static constexpr int kStageBytes = kSub * kSubBytes;
+    static constexpr int kStages = D == 128 ? (MB == 2 ? 4 : 5) : 6;
+    static constexpr int kBarBytes = 2048;
+    static constexpr int kRingDepth = 4;                       // hand-over slots between a row's column slices
+    static constexpr int kRings = 12;                          // (row block, warp quad, follower slice) triples, at most
+    static constexpr int kCombBytes = kRings * kRingDepth * 32 * 2 * 4;   // [ring][slot][lane][m, z]
+    static constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kBarBytes + kCombBytes + 1024;
+    static constexpr int kSlices = 4 / MB;                     // column slices of a tile, one per epilogue warp group
+    static constexpr int kEpiWarps = 16;
+    static constexpr int kThreads = 128 + kEpiWarps * 32;      // producer, two MMA issuers, one idle warp; epilogue
+};
+
+namespace tc {
+
+constexpr float kRefShift = 32.f;        // the first tile's row maximum is exponentiated to 2^-32
+constexpr float kRedoAbove = 1e30f;      // a partial sum at or above this sends its item to the exact kernel
+
+// 2^x on the FMA pipe for two values at a time (packed fp32 pairs), x clamped to [-125, 128].
+// The packed multiply-adds take one issue slot for two columns, which is what makes room for
+// this path beside the special-function one.
+__device__ __forceinline__ uint64_t exp2_fma2(uint64_t x2) {
+    float xa, xb;
+    unpack2(x2, xa, xb);
+    xa = fminf(fmaxf(xa, -125.f), 128.f);
+    xb = fminf(fmaxf(xb, -125.f), 128.f);
+    const uint64_t xc = pack2(xa, xb);
+    const uint64_t t = fadd2(xc, pack2(12582912.f, 12582912.f));       // 1.5 * 2^23: the low mantissa bits hold round(x)
+    const uint64_t fl = fadd2(t, pack2(-12582912.f, -12582912.f));
+    const uint64_t f = ffma2(fl, pack2(-1.f, -1.f), xc);                // in [-1/2, 1/2]
+    uint64_t q = ffma2(pack2(5.5171668e-02f, 5.5171668e-02f), f, pack2(2.4261112e-01f, 2.4261112e-01f));
+    q = ffma2(q, f, pack2(6.9326099e-01f, 6.9326099e-01f));
+    q = ffma2(q, f, pack2(9.9992807e-01f, 9.9992807e-01f));
+    float qa, qb, ta, tb;
+    unpack2(q, qa, qb);
+    unpack2(t, ta, tb);
+    return pack2(__uint_as_float(__float_as_uint(qa) + (__float_as_uint(ta) << 23)),
+                 __uint_as_float(__float_as_uint(qb) + (__float_as_uint(tb) << 23)));
+}
+
+// Is column pair j (of 16) of a 32-column chunk exponentiated on the FMA pipe?  NP pairs are, spread evenly.
+template <int NP>
+__device__ __forceinline__ constexpr bool pair_on_fma(int j) {
+    return NP > 0 && ((j + 1) * NP) / 16 != (j * NP) / 16;
+}
+
+// 2^(r[i] * scale + neg) for the column pair (2j, 2j+1), packed
+template <int NP>
+__device__ __forceinline__ uint64_t exp_pair(const uint32_t (&r)[32], int j, uint64_t sc2, uint64_t ng2) {
+    const uint64_t x2 = ffma2(pack2(SKV_F(r, 2 * j), SKV_F(r, 2 * j + 1)), sc2, ng2);
+    if (pair_on_fma<NP>(j)) return exp2_fma2(x2);
+    float xa, xb;
+    unpack2(x2, xa, xb);
+    return pack2(ex2f(xa), ex2f(xb));
+}
+
+// z[0..1] (packed pairs: four running sums) += 2^(r[i] * scale + neg) over the 32 columns
+template <int NP>
+__device__ __forceinline__ void expacc32(const uint32_t (&r)[32], float scale, float neg, uint64_t (&z)[2]) {
+    const uint64_t sc2 = pack2(scale, scale), ng2 = pack2(neg, neg);
+#pragma unroll
+    for (int j = 0; j < 16; ++j) z[j & 1] = fadd2(z[j & 1], exp_pair<NP>(r, j, sc2, ng2));
+}
+
+// r[i] = 2^(r[i] * scale + neg) in place, the same split between the two pipes
+template <int NP>
+__device__ __forceinline__ void exp32_mixed(uint32_t (&r)[32], float scale, float neg) {
+    const uint64_t sc2 = pack2(scale, scale), ng2 = pack2(neg, neg);
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        float ea, eb;
+        unpack2(exp_pair<NP>(r, j, sc2, ng2), ea, eb);
+        r[2 * j] = __float_as_uint(ea);
+        r[2 * j + 1] = __float_as_uint(eb);
+    }
+}
+
+}  // namespace tc
+
+template <int D, int MB, int PE>
+__global__ void __launch_bounds__(ScoreFastCfg<D, MB>::kThreads, 1)
+    score_fast_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const int q_box_rows,
+                      const int k_box_rows, const ScoreTcParams p) {
+    using Cfg = ScoreFastCfg<D, MB>;
+    constexpr int TN = tc::kTileKeys;
+    constexpr int NSL = Cfg::kSlices, SLW = TN / NSL, NCH = SLW / 32, RD = Cfg::kRingDepth;
+    extern __shared__ unsigned char smem_raw[];
+    tc::Pipe<Cfg> pp;
+    tc::pipe_setup(pp, smem_raw, Cfg::kEpiWarps / MB, Cfg::kRings * Cfg::kRingDepth * 2, 2);
+    float* comb = tc::pipe_scratch(pp, smem_raw);     // [ring][slot][lane][m, z]
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long total = p.total_items;
+    const int item_begin = (int)(total * blockIdx.x / gridDim.x);
+    const int item_end = (int)(total * (blockIdx.x + 1) / gridDim.x);
+
+    if (warp == 0) {
+        if (lane == 0) tc::producer_role<D, MB, false>(pp, &tmQ, &tmK, q_box_rows, k_box_rows, p, item_begin, item_end);
+    } else if (warp == 1 || warp == 2) {
+        if (lane == 0) tc::mma_role<D, MB, false, 2>(pp, p, item_begin, item_end, warp - 1);
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------------ epilogue
+        // a warp may touch the 32 tensor-memory lanes given by its index modulo 4; any four
+        // consecutive warps cover all 128 rows of a block
+        const int g = (warp - 4) >> 2, quad = warp & 3;
+        const int blk = MB == 2 ? (g >> 1) : 0;            // 128-row block of Q
+        const int slice = MB == 2 ? (g & 1) : g;           // column slice of every tile
+        const int lrow = quad * 32 + lane;
+        const int row = blk * 128 + lrow;
+        const bool live = row < p.R;                       // padding rows: their Q was never loaded
+        const int plim = live ? p.N - p.W + (row % p.W) : p.N - 1;
+        const float scale = p.scale_log2;
+        const int units_per_prompt = p.L * p.Hkv;
+        int acc = 0, nflush = 0;
+        uint32_t tfphase0 = 0, tfphase1 = 0;
+        bool ok = true;
+        for (int it = item_begin; it < item_end && ok; ++it) {
+            const int u = it / p.nchunk, j = it - u * p.nchunk;
+            const int lo = j * p.chunk_keys, hi = min(p.N, lo + p.chunk_keys);
+            const int nt = (hi - lo + TN - 1) / TN;
+            const int bprompt = u / units_per_prompt;
+            const int2* pcs = p.pieces + (size_t)bprompt * p.P;
+            int pi = p.chunk_first[(size_t)bprompt * p.cf_stride + j];
+            const int pi_last = p.chunk_first[(size_t)bprompt * p.cf_stride + j + 1];
+            // end of the current piece, and of the one after it: fetched one piece ahead so that the
+            // load's latency never sits between a piece end and the next comparison
+            int pend = pi < pi_last ? pcs[pi].y : 0x7fffffff;
+            int pend_n = pi + 1 < pi_last ? pcs[pi + 1].y : 0x7fffffff;
+            float m_ref = SHOTKV_NEG_INF, neg = 0.f;       // reference exponent of this (row, slice, item); neg = -m_ref
+            uint64_t z[2] = {0ull, 0ull};                  // four running sums of the current piece, as two packed pairs
+            const int plain_end = min(hi, p.N - p.W + 1);  // keys below this count for every window row
+
+            // piece `pi` is complete for this thread's columns.  A follower (slice > 0) posts its (m, z)
+            // in the next slot of its ring; the leader (slice 0) collects one slot from every follower
+            // of its rows, merges, and writes the piece's partials.
+            auto flush = [&]() {
+                float zz;
+                {
+                    float s0, s1, s2, s3;
+                    tc::unpack2(z[0], s0, s1);
+                    tc::unpack2(z[1], s2, s3);
+                    zz = (s0 + s1) + (s2 + s3);
+                }
+                const int slot = nflush & (RD - 1);
+                const uint32_t par = (uint32_t)(nflush / RD) & 1u;
+                if (slice != 0) {
+                    const int ring = (blk * 4 + quad) * (NSL - 1) + (slice - 1);
+                    const int rs = ring * RD + slot;
+                    if (nflush >= RD) {                                   // the slot's previous contents must have been read
+                        bool w = lane == 0 ? tc::mbar_wait(pp.extra_bar(rs * 2 + 1), par ^ 1u, pp.abort_flag, p.err) : true;
+                        w = __shfl_sync(0xffffffffu, w, 0);
+                        __syncwarp();
+                        ok = ok && w;
+                    }
+                    float2* dst = reinterpret_cast<float2*>(comb) + rs * 32 + lane;
+                    *dst = make_float2(m_ref, zz);
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(pp.extra_bar(rs * 2));
+                } else {
+                    float mm = m_ref, ms[NSL > 1 ? NSL - 1 : 1], zs[NSL > 1 ? NSL - 1 : 1];
+#pragma unroll
+                    for (int s = 1; s < NSL; ++s) {
+                        const int rs = ((blk * 4 + quad) * (NSL - 1) + (s - 1)) * RD + slot;
+                        bool w = lane == 0 ? tc::mbar_wait(pp.extra_bar(rs * 2), par, pp.abort_flag, p.err) : true;
+                        w = __shfl_sync(0xffffffffu, w, 0);
+                        __syncwarp();                                     // orders the other lanes' reads after lane 0's wait
+                        ok = ok && w;
+                        const float2 v = reinterpret_cast<const float2*>(comb)[rs * 32 + lane];
+                        __syncwarp();
+                        if (lane == 0) tc::mbar_arrive(pp.extra_bar(rs * 2 + 1));
+                        ms[s - 1] = v.x;
+                        zs[s - 1] = v.y;
+                        mm = fmaxf(mm, v.x);
+                    }
+                    const float mu = mm == SHOTKV_NEG_INF ? 0.f : mm;
+                    if (NSL > 1) zz *= ex2f(m_ref - mu);
+#pragma unroll
+                    for (int s = 1; s < NSL; ++s) zz += zs[s - 1] * ex2f(ms[s - 1] - mu);
+                    const size_t o = ((size_t)u * p.P + pi) * p.Rpad + row;
+                    p.part_m[o] = live ? mm : 0.f;
+                    p.part_z[o] = live ? zz : 0.f;
+                    if (live && !(zz < tc::kRedoAbove)) {  // out of range (or not a number): the exact kernel redoes the item
+                        p.redo[it] = 1;
+                        *p.redo_any = 1;
+                    }
+                }
+                z[0] = z[1] = 0ull;
+                ++nflush;
+                ++pi;
+                pend = pend_n;
+                pend_n = pi + 1 < pi_last ? pcs[pi + 1].y : 0x7fffffff;
+            };
+
+            // 32 columns starting at key kc0 that hold the end of the keys, the causal window, or a piece end
+            auto chunk_slow = [&](uint32_t (&r)[32], int kc0) {
+                while (pend <= kc0) flush();
+                if (kc0 + 32 <= plain_end && pend_n >= kc0 + 32) {
+                    // every column counts; at most one piece ends inside: one predicated pass
+                    tc::exp32_mixed<PE>(r, scale, neg);
+                    float lo_s, hi_s;
+                    tc::split32(r, min(pend - kc0, 32), lo_s, hi_s);
+                    z[0] = tc::fadd2(z[0], tc::pack2(lo_s, 0.f));
+                    if (pend < kc0 + 32) flush();
+                    z[0] = tc::fadd2(z[0], tc::pack2(hi_s, 0.f));
+                    return;
+                }
+                const int lim = min(hi, plim + 1) - kc0;                 // columns of the chunk that count
+                if (!__all_sync(0xffffffffu, lim >= 32)) tc::mask32(r, lim);
+                tc::exp32(r, scale, neg);
+                int start = 0;
+                while (pend < kc0 + 32) {
+                    const int e = pend - kc0;
+                    z[0] = tc::fadd2(z[0], tc::pack2(tc::range32(r, start, e), 0.f));
+                    start = e;
+                    flush();
+                }
+                z[0] = tc::fadd2(z[0], tc::pack2(tc::range32(r, start, 32), 0.f));
+            };
+
+            for (int t = 0; t < nt; ++t) {
+                const uint32_t tph = acc ? tfphase1 : tfphase0;
+                bool w = lane == 0 ? tc::mbar_wait(pp.tfull(acc, blk), tph, pp.abort_flag, p.err) : true;   // one poller per warp
+                w = __shfl_sync(0xffffffffu, w, 0);
+                if (!w || !ok) {
+                    ok = false;
+                    break;
+                }
+                if (acc) tfphase1 ^= 1; else tfphase0 ^= 1;
+                tc::fence_after_sync();
+                const int kc0 = lo + t * TN + slice * SLW;
+                const uint32_t taddr = pp.tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)((acc * MB + blk) * TN + slice * SLW);
+                uint32_t r[32];
+                if (t == 0) {
+                    // the item's reference exponent: this thread's maximum over its slice of the first tile
+                    float cm = SHOTKV_NEG_INF;
+#pragma unroll 1
+                    for (int c = 0; c < NCH; ++c) {
+                        tc::tmem_ld32_sync(r, taddr + c * 32);
+                        const int lim = min(hi, plim + 1) - (kc0 + c * 32);
+                        if (!__all_sync(0xffffffffu, lim >= 32)) tc::mask32(r, lim);
+                        cm = fmaxf(cm, tc::max32(r));
+                    }
+                    if (cm != SHOTKV_NEG_INF) {
+                        m_ref = fmaf(cm, scale, tc::kRefShift);
+                        neg = -m_ref;
+                    }
+                }
+#pragma unroll 1
+                for (int c = 0; c < NCH; ++c) {
+                    tc::tmem_ld32_sync(r, taddr + c * 32);
+                    if (c == NCH - 1) {                                   // the last of this tile's accumulators are in registers
+                        tc::fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) tc::mbar_arrive(pp.tempty(acc, blk));
+                    }
+                    // most chunks: every column counts for every row (it lies before the item's end and
+                    // before the first window position) and no piece ends at or inside the chunk
+                    if (kc0 + c * 32 + 32 <= min(pend, plain_end)) tc::expacc32<PE>(r, scale, neg, z);
+                    else chunk_slow(r, kc0 + c * 32);
+                }
+                acc ^= 1;
+            }
+            if (!ok) break;
+            while (pi < pi_last) flush();
+        }
+    }
+
+    tc::fence_before_sync();
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        tc::fence_after_sync();
+        tc::tmem_dealloc(pp.tmem_base, 512);
+    }
+}
+
+}  // namespace shotkv

@@ -40,6 +40,12 @@ struct ScoreTcParams {
     float* part_m;        // [U][P][Rpad]
     float* part_z;        // [U][P][Rpad]
     int* err;             // error word (host-visible); set to 1 when a bounded wait gave up
+    // Item filter.  The fast kernel (score_fast.cuh) raises redo[item] and *redo_any when an item's
+    // sums left the fp32 range it works in; the exact kernel, given the same arrays, recomputes
+    // only those items and returns at once when there is none.  Both NULL: every item is done.
+    int* redo;            // [total_items]
+    int* redo_any;
+    int* repaired;        // host-visible count of items recomputed under the filter (diagnostic)
 };
 
 template <int D, int MB>
@@ -299,6 +305,190 @@ __device__ __forceinline__ float range32(const uint32_t (&e)[32], int a, int b) 
     return s0 + s1;
 }
 
+
+
+// ---- the parts both scoring kernels share: shared-memory map, TMA producer, MMA issuer -------
+template <class Cfg>
+struct Pipe {
+    static constexpr int NST = Cfg::kStages;
+    uint32_t sQ, sK, sBar;      // shared-memory addresses: window queries, K stage ring, barriers
+    uint32_t tmem_base;
+    volatile int* abort_flag;
+    __device__ __forceinline__ uint32_t full(int s) const { return sBar + 8u * s; }
+    __device__ __forceinline__ uint32_t empty(int s) const { return sBar + 8u * (NST + s); }
+    __device__ __forceinline__ uint32_t qfull() const { return sBar + 8u * (2 * NST); }
+    __device__ __forceinline__ uint32_t qempty() const { return sBar + 8u * (2 * NST + 1); }
+    // accumulator-ready / accumulator-free barriers per (buffer, row block): the two row blocks of a
+    // tile are handed over separately
+    __device__ __forceinline__ uint32_t tfull(int a, int b) const { return sBar + 8u * (2 * NST + 2 + a * 2 + b); }
+    __device__ __forceinline__ uint32_t tempty(int a, int b) const { return sBar + 8u * (2 * NST + 6 + a * 2 + b); }
+    __device__ __forceinline__ uint32_t tmem_slot() const { return sBar + 8u * (2 * NST + 10); }
+    __device__ __forceinline__ uint32_t extra_bar(int i) const { return sBar + 256u + 8u * i; }
+};
+
+// Barrier set-up, tensor-memory allocation and the CTA-wide hand-over of its address.  Called by
+// every thread; `tempty_arrivals` = epilogue warps that release one (buffer, row block).
+// `extra` further barriers of one arrival each are initialised from pp.extra_bar(0) on.
+// `mma_threads` = threads running mma_role (each commits once to the Q-free barrier per unit).
+template <class Cfg>
+__device__ __forceinline__ void pipe_setup(Pipe<Cfg>& pp, unsigned char* smem_raw, int tempty_arrivals, int extra = 0,
+                                           int mma_threads = 1) {
+    constexpr int NST = Cfg::kStages;
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;
+    unsigned char* gbase = smem_raw + (base - raw_addr);
+    pp.sQ = base;
+    pp.sK = base + Cfg::kQBytes;
+    pp.sBar = pp.sK + NST * Cfg::kStageBytes;
+    volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(gbase + (pp.tmem_slot() - base));
+    pp.abort_flag = reinterpret_cast<volatile int*>(gbase + (pp.tmem_slot() - base) + 4);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NST; ++s) {
+            mbar_init(pp.full(s), 1);
+            mbar_init(pp.empty(s), 1);
+        }
+        mbar_init(pp.qfull(), 1);
+        mbar_init(pp.qempty(), mma_threads);
+        for (int a = 0; a < 2; ++a)
+            for (int b = 0; b < 2; ++b) {
+                mbar_init(pp.tfull(a, b), 1);
+                mbar_init(pp.tempty(a, b), tempty_arrivals);
+            }
+        for (int i = 0; i < extra; ++i) mbar_init(pp.extra_bar(i), 1);
+        *pp.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if ((threadIdx.x >> 5) == 0) {
+        tmem_alloc(pp.tmem_slot(), 512);
+        tmem_relinquish();
+    }
+    fence_before_sync();
+    __syncthreads();
+    fence_after_sync();
+    pp.tmem_base = *tmem_slot_g;
+}
+// The scratch area behind the barriers (merging of a row's column slices).
+template <class Cfg>
+__device__ __forceinline__ float* pipe_scratch(const Pipe<Cfg>& pp, unsigned char* smem_raw) {
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    return reinterpret_cast<float*>(smem_raw + (pp.sBar - raw_addr) + Cfg::kBarBytes);
+}
+
+// One thread: the unit's window queries (once per unit) and K tiles of 128 keys into the ring.
+// FILTERED: skip the items whose redo flag is clear (the exact kernel's repair launches).
+template <int D, int MB, bool FILTERED, class Cfg>
+__device__ __forceinline__ void producer_role(const Pipe<Cfg>& pp, const CUtensorMap* tmQ, const CUtensorMap* tmK,
+                                              int q_box_rows, int k_box_rows, const ScoreTcParams& p, int item_begin,
+                                              int item_end) {
+    constexpr int NSUB = Cfg::kSub, NST = Cfg::kStages, TN = kTileKeys;
+    int stage = 0, cur_u = -1, outstanding = 0;
+    uint32_t ephase = 1, qephase = 1;
+    bool ok = true;
+    for (int it = item_begin; it < item_end && ok; ++it) {
+        if (FILTERED && p.redo && !p.redo[it]) continue;
+        const int u = it / p.nchunk, j = it - u * p.nchunk;
+        const int lo = j * p.chunk_keys, hi = min(p.N, lo + p.chunk_keys);
+        const int nt = (hi - lo + TN - 1) / TN;
+        if (nt <= 0) continue;
+        if (u != cur_u) {
+            if (!(ok = mbar_wait_relaxed(pp.qempty(), qephase, pp.abort_flag, p.err))) break;
+            qephase ^= 1;
+            mbar_expect_tx(pp.qfull(), MB * NSUB * q_box_rows * 128);
+#pragma unroll
+            for (int b = 0; b < MB; ++b)
+#pragma unroll
+                for (int sub = 0; sub < NSUB; ++sub)
+                    tma_load_2d(pp.sQ + (b * NSUB + sub) * Cfg::kSubBytes, tmQ, sub * 64, u * p.R + b * 128, pp.qfull());
+            cur_u = u;
+        }
+        for (int t = 0; t < nt; ++t) {
+            if (!(ok = mbar_wait_relaxed(pp.empty(stage), ephase, pp.abort_flag, p.err))) break;
+            mbar_expect_tx(pp.full(stage), NSUB * k_box_rows * 128);
+#pragma unroll
+            for (int sub = 0; sub < NSUB; ++sub)
+                tma_load_3d(pp.sK + stage * Cfg::kStageBytes + sub * Cfg::kSubBytes, tmK, sub * 64, lo + t * TN, u, pp.full(stage));
+            outstanding = outstanding < NST ? outstanding + 1 : NST;
+            if (++stage == NST) {
+                stage = 0;
+                ephase ^= 1;
+            }
+        }
+    }
+    if (!ok) {
+        // aborting: give the copies already issued a bounded time to land before the CTA ends
+        const long long t0 = clock64();
+        int s = stage;
+        uint32_t ph = ephase;
+        for (int k = 0; k < outstanding; ++k) {
+            if (--s < 0) {
+                s = NST - 1;
+                ph ^= 1;
+            }
+            while (!mbar_try(pp.full(s), ph ^ 1) && clock64() - t0 < kWaitCycles) {
+            }
+        }
+    }
+}
+
+// S[128 x 128] = Q_block . K_tile^T per 128-row block of Q, fp32 accumulators double-buffered in
+// tensor memory (buffer a, row block b at column (a * MB + b) * 128).  Run by NT threads of
+// different warps; thread `which` issues the tiles whose running index is `which` modulo NT.
+// With NT = 2 each thread owns one accumulator buffer, so the two never touch the same barriers
+// except the K-stage ring (each waits for and frees the stages of its own tiles) and the Q pair.
+// A lone issuing thread shares its scheduler with four epilogue warps that seldom stall, and is
+// selected so rarely that sixteen MMAs per tile take it longer than the tile's epilogue.
+template <int D, int MB, bool FILTERED, int NT, class Cfg>
+__device__ __forceinline__ void mma_role(const Pipe<Cfg>& pp, const ScoreTcParams& p, int item_begin, int item_end,
+                                         int which) {
+    constexpr int NSUB = Cfg::kSub, KSTEPS = D / 16, NST = Cfg::kStages, TN = kTileKeys;
+    constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TN >> 3) << 17) | ((128u >> 4) << 24);
+    int stage = 0, acc = 0, cur_u = -1;
+    uint32_t fphase = 0, qfphase = 0, tephase0 = 1, tephase1 = 1;
+    bool ok = true;
+    for (int it = item_begin; it < item_end && ok; ++it) {
+        if (FILTERED && p.redo && !p.redo[it]) continue;
+        const int u = it / p.nchunk, j = it - u * p.nchunk;
+        const int lo = j * p.chunk_keys, hi = min(p.N, lo + p.chunk_keys);
+        const int nt = (hi - lo + TN - 1) / TN;
+        if (nt <= 0) continue;
+        if (u != cur_u) {
+            if (cur_u >= 0) umma_commit(pp.qempty());     // Q may be replaced once these MMAs are done
+            if (!(ok = mbar_wait_relaxed(pp.qfull(), qfphase, pp.abort_flag, p.err))) break;
+            qfphase ^= 1;
+            cur_u = u;
+        }
+        for (int t = 0; t < nt; ++t) {
+            const bool mine = NT == 1 || acc == which;
+            if (mine) {
+            if (!(ok = mbar_wait_relaxed(pp.full(stage), fphase, pp.abort_flag, p.err))) break;
+            const uint32_t tph = acc ? tephase1 : tephase0;
+            const uint32_t kb = pp.sK + stage * Cfg::kStageBytes;
+#pragma unroll
+            for (int b = 0; b < MB; ++b) {
+                if (!(ok = mbar_wait_relaxed(pp.tempty(acc, b), tph, pp.abort_flag, p.err))) break;
+                fence_after_sync();
+                const uint32_t d_tmem = pp.tmem_base + (uint32_t)((acc * MB + b) * TN);
+#pragma unroll
+                for (int ks = 0; ks < KSTEPS; ++ks) {
+                    const uint32_t a_addr = pp.sQ + (b * NSUB + (ks >> 2)) * Cfg::kSubBytes + (ks & 3) * 32;
+                    const uint32_t b_addr = kb + (ks >> 2) * Cfg::kSubBytes + (ks & 3) * 32;
+                    umma_bf16(d_tmem, smem_desc(a_addr), smem_desc(b_addr), idesc, ks > 0);
+                }
+                umma_commit(pp.tfull(acc, b));
+            }
+            if (!ok) break;
+            if (acc) tephase1 ^= 1; else tephase0 ^= 1;
+            umma_commit(pp.empty(stage));
+            }
+            if (++stage == NST) {
+                stage = 0;
+                fphase ^= 1;
+            }
+            acc ^= 1;
+        }
+    }
+}
+
 }  // namespace tc
 
 template <int D, int MB>
@@ -306,152 +496,27 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
     score_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const int q_box_rows,
                     const int k_box_rows, const ScoreTcParams p) {
     using Cfg = ScoreTcCfg<D, MB>;
-    constexpr int NSUB = Cfg::kSub, KSTEPS = D / 16, NST = Cfg::kStages, TN = tc::kTileKeys;
+    constexpr int TN = tc::kTileKeys;
     constexpr int NSL = Cfg::kSlices, SLW = TN / NSL, NCH = SLW / 32;     // slices, slice width, chunks per slice
     extern __shared__ unsigned char smem_raw[];
-    const uint32_t raw_addr = smem_u32(smem_raw);
-    const uint32_t base = (raw_addr + 1023u) & ~1023u;
-    unsigned char* gbase = smem_raw + (base - raw_addr);
-    const uint32_t sQ = base, sK = base + Cfg::kQBytes, sBar = sK + NST * Cfg::kStageBytes;
-    auto bar_full = [&](int s) { return sBar + 8u * s; };
-    auto bar_empty = [&](int s) { return sBar + 8u * (NST + s); };
-    const uint32_t bar_qfull = sBar + 8u * (2 * NST), bar_qempty = bar_qfull + 8u;
-    // accumulator-ready / accumulator-free barriers per (buffer, row block): the two row blocks of a
-    // tile are handed over separately, which keeps their epilogue warps half a chunk out of phase
-    auto bar_tfull = [&](int a, int b) { return sBar + 8u * (2 * NST + 2 + a * 2 + b); };
-    auto bar_tempty = [&](int a, int b) { return sBar + 8u * (2 * NST + 6 + a * 2 + b); };
-    const uint32_t tmem_slot = sBar + 8u * (2 * NST + 10);
-    volatile uint32_t* tmem_slot_g = reinterpret_cast<volatile uint32_t*>(gbase + (tmem_slot - base));
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + (tmem_slot - base) + 4);
-    float* comb = reinterpret_cast<float*>(gbase + (sBar - base) + Cfg::kBarBytes);   // [2][4][128][2]
+    if (p.redo_any && *p.redo_any == 0) return;       // repair launch with nothing to repair
+    tc::Pipe<Cfg> pp;
+    tc::pipe_setup(pp, smem_raw, 16 / MB);
+    float* comb = tc::pipe_scratch(pp, smem_raw);     // [2][4][128][2]
+    const uint32_t tmem_base = pp.tmem_base;
+    volatile int* abort_flag = pp.abort_flag;
+    auto bar_tfull = [&](int a, int b) { return pp.tfull(a, b); };
+    auto bar_tempty = [&](int a, int b) { return pp.tempty(a, b); };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < NST; ++s) {
-            tc::mbar_init(bar_full(s), 1);
-            tc::mbar_init(bar_empty(s), 1);
-        }
-        tc::mbar_init(bar_qfull, 1);
-        tc::mbar_init(bar_qempty, 1);
-        for (int a = 0; a < 2; ++a)
-            for (int b = 0; b < 2; ++b) {
-                tc::mbar_init(bar_tfull(a, b), 1);
-                tc::mbar_init(bar_tempty(a, b), 16 / MB);     // one arrival per epilogue warp of the row block
-            }
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == 0) {
-        tc::tmem_alloc(tmem_slot, 512);
-        tc::tmem_relinquish();
-    }
-    tc::fence_before_sync();
-    __syncthreads();
-    tc::fence_after_sync();
-    const uint32_t tmem_base = *tmem_slot_g;
-
     const long long total = p.total_items;
     const int item_begin = (int)(total * blockIdx.x / gridDim.x);
     const int item_end = (int)(total * (blockIdx.x + 1) / gridDim.x);
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            int stage = 0, cur_u = -1, outstanding = 0;
-            uint32_t ephase = 1, qephase = 1;
-            bool ok = true;
-            for (int it = item_begin; it < item_end && ok; ++it) {
-                const int u = it / p.nchunk, j = it - u * p.nchunk;
-                const int lo = j * p.chunk_keys, hi = min(p.N, lo + p.chunk_keys);
-                const int nt = (hi - lo + TN - 1) / TN;
-                if (nt <= 0) continue;
-                if (u != cur_u) {
-                    if (!(ok = tc::mbar_wait_relaxed(bar_qempty, qephase, abort_flag, p.err))) break;
-                    qephase ^= 1;
-                    tc::mbar_expect_tx(bar_qfull, MB * NSUB * q_box_rows * 128);
-#pragma unroll
-                    for (int b = 0; b < MB; ++b)
-#pragma unroll
-                        for (int sub = 0; sub < NSUB; ++sub)
-                            tc::tma_load_2d(sQ + (b * NSUB + sub) * Cfg::kSubBytes, &tmQ, sub * 64, u * p.R + b * 128, bar_qfull);
-                    cur_u = u;
-                }
-                for (int t = 0; t < nt; ++t) {
-                    if (!(ok = tc::mbar_wait_relaxed(bar_empty(stage), ephase, abort_flag, p.err))) break;
-                    tc::mbar_expect_tx(bar_full(stage), NSUB * k_box_rows * 128);
-#pragma unroll
-                    for (int sub = 0; sub < NSUB; ++sub)
-                        tc::tma_load_3d(sK + stage * Cfg::kStageBytes + sub * Cfg::kSubBytes, &tmK, sub * 64, lo + t * TN, u,
-                                        bar_full(stage));
-                    outstanding = outstanding < NST ? outstanding + 1 : NST;
-                    if (++stage == NST) {
-                        stage = 0;
-                        ephase ^= 1;
-                    }
-                }
-            }
-            if (!ok) {
-                // aborting: give the copies already issued a bounded time to land before the CTA ends
-                const long long t0 = clock64();
-                int s = stage;
-                uint32_t ph = ephase;
-                for (int k = 0; k < outstanding; ++k) {
-                    if (--s < 0) {
-                        s = NST - 1;
-                        ph ^= 1;
-                    }
-                    while (!tc::mbar_try(bar_full(s), ph ^ 1) && clock64() - t0 < tc::kWaitCycles) {
-                    }
-                }
-            }
-        }
+        if (lane == 0) tc::producer_role<D, MB, true>(pp, &tmQ, &tmK, q_box_rows, k_box_rows, p, item_begin, item_end);
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TN >> 3) << 17) | ((128u >> 4) << 24);
-            int stage = 0, acc = 0, cur_u = -1;
-            uint32_t fphase = 0, qfphase = 0, tephase0 = 1, tephase1 = 1;
-            bool ok = true;
-            for (int it = item_begin; it < item_end && ok; ++it) {
-                const int u = it / p.nchunk, j = it - u * p.nchunk;
-                const int lo = j * p.chunk_keys, hi = min(p.N, lo + p.chunk_keys);
-                const int nt = (hi - lo + TN - 1) / TN;
-                if (nt <= 0) continue;
-                if (u != cur_u) {
-                    if (cur_u >= 0) tc::umma_commit(bar_qempty);     // Q may be replaced once these MMAs are done
-                    if (!(ok = tc::mbar_wait_relaxed(bar_qfull, qfphase, abort_flag, p.err))) break;
-                    qfphase ^= 1;
-                    cur_u = u;
-                }
-                for (int t = 0; t < nt; ++t) {
-                    if (!(ok = tc::mbar_wait_relaxed(bar_full(stage), fphase, abort_flag, p.err))) break;
-                    const uint32_t tph = acc ? tephase1 : tephase0;
-                    const uint32_t kb = sK + stage * Cfg::kStageBytes;
-#pragma unroll
-                    for (int b = 0; b < MB; ++b) {
-                        if (!(ok = tc::mbar_wait_relaxed(bar_tempty(acc, b), tph, abort_flag, p.err))) break;
-                        tc::fence_after_sync();
-                        const uint32_t d_tmem = tmem_base + (uint32_t)((acc * MB + b) * TN);
-#pragma unroll
-                        for (int ks = 0; ks < KSTEPS; ++ks) {
-                            const uint32_t a_addr = sQ + (b * NSUB + (ks >> 2)) * Cfg::kSubBytes + (ks & 3) * 32;
-                            const uint32_t b_addr = kb + (ks >> 2) * Cfg::kSubBytes + (ks & 3) * 32;
-                            tc::umma_bf16(d_tmem, tc::smem_desc(a_addr), tc::smem_desc(b_addr), idesc, ks > 0);
-                        }
-                        tc::umma_commit(bar_tfull(acc, b));
-                    }
-                    if (!ok) break;
-                    if (acc) tephase1 ^= 1; else tephase0 ^= 1;
-                    tc::umma_commit(bar_empty(stage));
-                    if (++stage == NST) {
-                        stage = 0;
-                        fphase ^= 1;
-                    }
-                    acc ^= 1;
-                }
-            }
-        }
+        if (lane == 0) tc::mma_role<D, MB, true, 1>(pp, p, item_begin, item_end, 0);
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ epilogue
         // a warp may touch the 32 tensor-memory lanes given by its index modulo 4; any four
@@ -468,6 +533,10 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
         uint32_t tfphase0 = 0, tfphase1 = 0;
         bool ok = true;
         for (int it = item_begin; it < item_end && ok; ++it) {
+            if (p.redo) {
+                if (!p.redo[it]) continue;
+                if (warp == 4 && lane == 0) atomicAdd(p.repaired, 1);
+            }
             const int u = it / p.nchunk, j = it - u * p.nchunk;
             const int lo = j * p.chunk_keys, hi = min(p.N, lo + p.chunk_keys);
             const int nt = (hi - lo + TN - 1) / TN;

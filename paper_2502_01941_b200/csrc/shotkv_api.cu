@@ -14,6 +14,7 @@
 
 #include "common.cuh"
 #include "decode.cuh"
+#include "score_fast.cuh"
 #include "score_mma.cuh"
 #include "score_tc.cuh"
 #include "select_compact.cuh"
@@ -49,6 +50,7 @@ struct shotkv_ctx {
     int* err_host = nullptr;
     int* err_dev = nullptr;
     int sm_count = 148;
+    int scoring_mode = SHOTKV_SCORING_FAST;
 };
 
 namespace {
@@ -147,6 +149,7 @@ struct PrefillWs {
     float* row_m;      // [U][Rpad]
     float* row_invz;
     float* unit_shot;  // [U][S]
+    int* redo;         // [1 + U * kMaxChunks] word 0: some item is marked; then one word per item the exact kernel must recompute
     size_t total;
 };
 
@@ -164,6 +167,7 @@ PrefillWs carve(const shotkv_dims* d, void* base) {
     w.row_m = (float*)take(U * R * 4);
     w.row_invz = (float*)take(U * R * 4);
     w.unit_shot = (float*)take(U * (size_t)(d->S > 0 ? d->S : 1) * 4);
+    w.redo = (int*)take((U * kMaxChunks + 1) * 4);
     w.total = o;
     return w;
 }
@@ -331,6 +335,21 @@ int launch_score_tc_t(shotkv_ctx* ctx, const CUtensorMap& tmQ, const CUtensorMap
     return SHOTKV_OK;
 }
 
+// Column pairs, of every 16, whose exponentials run on the FMA pipe instead of the special-function unit.
+constexpr int kPolyEvery = 5;
+
+template <int D, int MB>
+int launch_score_fast_t(shotkv_ctx* ctx, const CUtensorMap& tmQ, const CUtensorMap& tmK, int qbox, int kbox,
+                        const ScoreTcParams& sp, cudaStream_t stream) {
+    constexpr int smem = ScoreFastCfg<D, MB>::kSmemBytes;
+    CUDA_TRY(ctx, cudaFuncSetAttribute(score_fast_kernel<D, MB, kPolyEvery>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    int grid = sp.total_items < ctx->sm_count ? sp.total_items : ctx->sm_count;
+    if (grid < 1) grid = 1;
+    score_fast_kernel<D, MB, kPolyEvery><<<grid, ScoreFastCfg<D, MB>::kThreads, smem, stream>>>(tmQ, tmK, qbox, kbox, sp);
+    LAUNCH_CHECK(ctx);
+    return SHOTKV_OK;
+}
+
 int launch_score_tc(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const shotkv_bf16* K, const PrefillWs& w,
                     int P, const ChunkPlan& plan, cudaStream_t stream) {
     EncodeTiledFn enc = encode_tiled_fn();
@@ -370,7 +389,19 @@ int launch_score_tc(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q,
     sp.scale_log2 = kLog2e / sqrtf((float)d->d);
     sp.part_m = w.part_m; sp.part_z = w.part_z;
     sp.err = ctx->err_dev;
+    sp.repaired = ctx->err_dev + 1;
     const bool big = sp.Rpad == 256;
+    int rc = SHOTKV_OK;
+    if (ctx->scoring_mode == SHOTKV_SCORING_FAST) {
+        // fast kernel first; it marks the items whose sums left its range, and the exact kernel
+        // below then redoes exactly those (returning at once when there is none)
+        sp.redo_any = w.redo;
+        sp.redo = w.redo + 1;
+        CUDA_TRY(ctx, cudaMemsetAsync(w.redo, 0, ((size_t)sp.total_items + 1) * 4, stream));
+        if (d->d == 128) rc = big ? launch_score_fast_t<128, 2>(ctx, tmQ, tmK, qbox, kbox, sp, stream) : launch_score_fast_t<128, 1>(ctx, tmQ, tmK, qbox, kbox, sp, stream);
+        else rc = big ? launch_score_fast_t<64, 2>(ctx, tmQ, tmK, qbox, kbox, sp, stream) : launch_score_fast_t<64, 1>(ctx, tmQ, tmK, qbox, kbox, sp, stream);
+        if (rc) return rc;
+    }
     if (d->d == 128) return big ? launch_score_tc_t<128, 2>(ctx, tmQ, tmK, qbox, kbox, sp, stream) : launch_score_tc_t<128, 1>(ctx, tmQ, tmK, qbox, kbox, sp, stream);
     return big ? launch_score_tc_t<64, 2>(ctx, tmQ, tmK, qbox, kbox, sp, stream) : launch_score_tc_t<64, 1>(ctx, tmQ, tmK, qbox, kbox, sp, stream);
 }
@@ -471,12 +502,13 @@ int shotkv_create(shotkv_ctx** out, int device) {
             delete ctx;
             return SHOTKV_ERR_CUDA;
         }
-    if (cudaHostAlloc((void**)&ctx->err_host, sizeof(int), cudaHostAllocMapped) != cudaSuccess ||
+    if (cudaHostAlloc((void**)&ctx->err_host, 2 * sizeof(int), cudaHostAllocMapped) != cudaSuccess ||
         cudaHostGetDevicePointer((void**)&ctx->err_dev, ctx->err_host, 0) != cudaSuccess) {
         shotkv_destroy(ctx);
         return SHOTKV_ERR_CUDA;
     }
-    *ctx->err_host = 0;
+    ctx->err_host[0] = 0;      // word 0: a bounded wait gave up
+    ctx->err_host[1] = 0;      // word 1: work items the exact scoring kernel recomputed after the fast one
     ctx->sm_count = prop.multiProcessorCount;
     *out = ctx;
     return SHOTKV_OK;
@@ -914,6 +946,14 @@ int32_t shotkv_plan_pieces(const shotkv_dims* dims, const int32_t* offsets_host,
 }
 
 // ---- instrumentation ------------------------------------------------------------------------
+int shotkv_set_scoring_mode(shotkv_ctx* ctx, int mode) {
+    if (!ctx) return SHOTKV_ERR_INVALID_ARG;
+    if (mode != SHOTKV_SCORING_FAST && mode != SHOTKV_SCORING_EXACT)
+        return fail(ctx, SHOTKV_ERR_INVALID_ARG, "scoring mode must be SHOTKV_SCORING_FAST or SHOTKV_SCORING_EXACT");
+    ctx->scoring_mode = mode;
+    return SHOTKV_OK;
+}
+
 int shotkv_profile_enable(shotkv_ctx* ctx, int enable) {
     int rc = set_device(ctx);
     if (rc) return rc;
@@ -941,5 +981,9 @@ int shotkv_profile_read(shotkv_ctx* ctx, int calls_back, float* stage_ms) {
 }
 
 uint64_t shotkv_launch_count(const shotkv_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+uint64_t shotkv_repaired_items(const shotkv_ctx* ctx) {
+    return ctx && ctx->err_host ? (uint64_t)(unsigned)((volatile int*)ctx->err_host)[1] : 0;
+}
 
 }  // extern "C"

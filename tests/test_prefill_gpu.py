@@ -270,3 +270,46 @@ def test_full_size_sampled_units(ctx, cid, units):
             assert torch.equal(gpu["Vc"][b, l, :, :n], V[b, l][:, idx[b, l, :n]])
     del Q, K, V, gpu
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("cfg", SHRUNK, ids=[c.name for c in SHRUNK])
+def test_exact_scoring_mode(ctx, cfg):
+    """The exact kernel alone (running maximum per row) gives the same parity as the default pair."""
+    skv.shotkv_set_scoring_mode(ctx, skv.SCORING_EXACT)
+    try:
+        ties, _ = run_cfg(ctx, cfg, "fused")
+    finally:
+        skv.shotkv_set_scoring_mode(ctx, skv.SCORING_FAST)
+    assert ties <= 2
+
+
+@pytest.mark.parametrize("col", [3, 6])
+def test_fast_scoring_out_of_range_items_are_recomputed(ctx, col):
+    """A key whose logit lies thousands of nats above its work item's first tile leaves the fp32
+    range the fast kernel works in (on the special-function path for col 6, on the FMA path for
+    col 3); the item must be recomputed by the exact kernel and the result must still match."""
+    cfg = wl.PrefillConfig("outlier", B=1, L=8, H=16, Hkv=8, d=64, N=2048, W=16, S=6, shot_dist="uniform", shot_lo=200,
+                           shot_hi=400, question_len=100, r_p=0.5, cfg_id=21)
+    Q, K, V, off = wl.prefill_batch(cfg, "cuda")
+    dims = P.dims_of(cfg)
+    Qd = Q.clone(); Qd[..., 0] = 8.0
+    Kd = K.clone(); Kd[..., 0] = 0.0
+    nchunk, chunk_keys, _ = skv.shotkv_plan_pieces(dims, off)
+    # a key in the second tile of the first work item, at a chosen column of its 32-column chunk
+    tstar = 128 + 32 + col
+    assert chunk_keys >= 256, "the case needs work items of at least two tiles"
+    s_hit = int(np.searchsorted(off[0], tstar, side="right")) - 1
+    assert 0 <= s_hit < cfg.S
+    Kd[0, 0, :, tstar, 0] = 2000.0            # layer 0 only: logit 8*2000/sqrt(64) = 2000
+    before = skv.shotkv_repaired_items(ctx)
+    gpu = P.gpu_prefill(ctx, dims, Qd, Kd, V, off, cfg.r_p, 0, "fused")
+    assert skv.shotkv_repaired_items(ctx) - before == cfg.Hkv          # layer 0: one item per kv head
+    sc = gpu["shot_scores"][0, 0].cpu().numpy()
+    k_hit = int(off[0, s_hit + 1] - off[0, s_hit])
+    np.testing.assert_allclose(sc[s_hit], cfg.H * cfg.W / k_hit, rtol=1e-4)
+    P.check_all_units(gpu, Qd, Kd, V, off, cfg.r_p)
+    # an ordinary input right after it needs no repair
+    before = skv.shotkv_repaired_items(ctx)
+    gpu = P.gpu_prefill(ctx, dims, Q, K, V, off, cfg.r_p, 0, "fused")
+    assert skv.shotkv_repaired_items(ctx) == before
+    P.check_all_units(gpu, Q, K, V, off, cfg.r_p)
