@@ -38,8 +38,8 @@ struct ScoreFastCfg {
     static constexpr int kRings = 12;                          // (row block, warp quad, follower slice) triples, at most
     static constexpr int kCombBytes = kRings * kRingDepth * 32 * 2 * 4;   // [ring][slot][lane][m, z]
     static constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kBarBytes + kCombBytes + 1024;
-    static constexpr int kSlices = 4 / MB;                     // column slices of a tile, one per epilogue warp group
-    static constexpr int kEpiWarps = 16;
+    static constexpr int kSlices = 2 / MB;                     // column slices of a tile
+    static constexpr int kEpiWarps = 8;
     static constexpr int kThreads = 128 + kEpiWarps * 32;      // producer, two MMA issuers, one idle warp; epilogue
 };
 
@@ -135,8 +135,8 @@ __global__ void __launch_bounds__(ScoreFastCfg<D, MB>::kThreads, 1)
         // a warp may touch the 32 tensor-memory lanes given by its index modulo 4; any four
         // consecutive warps cover all 128 rows of a block
         const int g = (warp - 4) >> 2, quad = warp & 3;
-        const int blk = MB == 2 ? (g >> 1) : 0;            // 128-row block of Q
-        const int slice = MB == 2 ? (g & 1) : g;           // column slice of every tile
+        const int blk = MB == 2 ? g : 0;                   // 128-row block of Q
+        const int slice = MB == 2 ? 0 : g;                 // column slice of every tile
         const int lrow = quad * 32 + lane;
         const int row = blk * 128 + lrow;
         const bool live = row < p.R;                       // padding rows: their Q was never loaded
@@ -251,12 +251,12 @@ __global__ void __launch_bounds__(ScoreFastCfg<D, MB>::kThreads, 1)
 
             for (int t = 0; t < nt; ++t) {
                 const uint32_t tph = acc ? tfphase1 : tfphase0;
-                bool w = lane == 0 ? tc::mbar_wait(pp.tfull(acc, blk), tph, pp.abort_flag, p.err) : true;   // one poller per warp
-                w = __shfl_sync(0xffffffffu, w, 0);
-                if (!w || !ok) {
-                    ok = false;
-                    break;
+                if (!tc::mbar_try(pp.tfull(acc, blk), tph)) {            // usually ready: one test by the whole warp
+                    bool w = lane == 0 ? tc::mbar_wait(pp.tfull(acc, blk), tph, pp.abort_flag, p.err) : true;   // one poller per warp
+                    w = __shfl_sync(0xffffffffu, w, 0);
+                    if (!w) ok = false;
                 }
+                if (!ok) break;
                 if (acc) tfphase1 ^= 1; else tfphase0 ^= 1;
                 tc::fence_after_sync();
                 const int kc0 = lo + t * TN + slice * SLW;
@@ -277,18 +277,29 @@ __global__ void __launch_bounds__(ScoreFastCfg<D, MB>::kThreads, 1)
                         neg = -m_ref;
                     }
                 }
+                auto release = [&]() {                                   // this tile's accumulators are all in registers
+                    tc::fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(pp.tempty(acc, blk));
+                };
+                if (kc0 + SLW <= min(pend, plain_end)) {
+                    // most tiles: every column of the slice counts for every row (it lies before the
+                    // item's end and before the first window position) and no piece ends inside it.
+                    // One short loop without further branches.
 #pragma unroll 1
-                for (int c = 0; c < NCH; ++c) {
-                    tc::tmem_ld32_sync(r, taddr + c * 32);
-                    if (c == NCH - 1) {                                   // the last of this tile's accumulators are in registers
-                        tc::fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) tc::mbar_arrive(pp.tempty(acc, blk));
+                    for (int c = 0; c < NCH; ++c) {
+                        tc::tmem_ld32_sync(r, taddr + c * 32);
+                        tc::expacc32<PE>(r, scale, neg, z);
                     }
-                    // most chunks: every column counts for every row (it lies before the item's end and
-                    // before the first window position) and no piece ends at or inside the chunk
-                    if (kc0 + c * 32 + 32 <= min(pend, plain_end)) tc::expacc32<PE>(r, scale, neg, z);
-                    else chunk_slow(r, kc0 + c * 32);
+                    release();
+                } else {
+#pragma unroll 1
+                    for (int c = 0; c < NCH; ++c) {
+                        tc::tmem_ld32_sync(r, taddr + c * 32);
+                        if (c == NCH - 1) release();
+                        if (kc0 + c * 32 + 32 <= min(pend, plain_end)) tc::expacc32<PE>(r, scale, neg, z);
+                        else chunk_slow(r, kc0 + c * 32);
+                    }
                 }
                 acc ^= 1;
             }
