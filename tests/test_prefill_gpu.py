@@ -295,9 +295,10 @@ def test_fast_scoring_out_of_range_items_are_recomputed(ctx, col):
     Qd = Q.clone(); Qd[..., 0] = 8.0
     Kd = K.clone(); Kd[..., 0] = 0.0
     nchunk, chunk_keys, _ = skv.shotkv_plan_pieces(dims, off)
-    # a key in the second tile of the first work item, at a chosen column of its 32-column chunk
-    tstar = 128 + 32 + col
-    assert chunk_keys >= 256, "the case needs work items of at least two tiles"
+    # a key in the fourth tile of the first work item (every epilogue warp set has fixed its reference
+    # on an earlier tile by then), at a chosen column of its 32-column chunk
+    tstar = 3 * 128 + 32 + col
+    assert chunk_keys >= 512, "the case needs work items of at least four tiles"
     s_hit = int(np.searchsorted(off[0], tstar, side="right")) - 1
     assert 0 <= s_hit < cfg.S
     Kd[0, 0, :, tstar, 0] = 2000.0            # layer 0 only: logit 8*2000/sqrt(64) = 2000
