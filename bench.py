@@ -42,8 +42,8 @@ METRIC = "prompt tokens compressed/sec"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the scoring kernel per algorithmic K byte, from the ncu capture summarised in
-# profiles/score_tc_kernel_cfg3_B1_L8.md; set to None whenever the kernel changes after the capture.
-SCORE_TC_TRAFFIC_RATIO = 1.043
+# profiles/score_fast_kernel_cfg3_B1_L8.md; set to None whenever the kernel changes after the capture.
+SCORE_TC_TRAFFIC_RATIO = 1.047
 DECODE_TRAFFIC_RATIO = 1.012    # profiles/decode_score_kernel_cfg4_B2.md
 NOMINAL_HBM_GBS = 8000.0
 
@@ -90,7 +90,7 @@ class ClockSampler:
         self.f.flush()
         self.f.seek(0)
         import datetime
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         for line in self.f.read().splitlines():
             parts = [x.strip() for x in line.split(",")]
             if len(parts) < 9:
@@ -100,6 +100,7 @@ class ClockSampler:
                 if t_begin is not None and not (t_begin - 0.05 <= ts <= t_end + 0.05):
                     continue
                 sm.append(float(parts[1])); mx.append(float(parts[2]))
+                pw.append(float(parts[3]))
             except ValueError:
                 continue
             for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[5:9]):
@@ -110,7 +111,7 @@ class ClockSampler:
         except OSError:
             pass
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "power_w": statistics.median(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
 def dist_setup(n_gpus: int):
@@ -215,16 +216,19 @@ def run_ours(args):
     logits = cfg.B * cfg.L * cfg.H * cfg.W * cfg.N                       # one ex2 per window logit
     sm_mhz = clocks.get("sm_mhz") or 1965.0
     ex2_rate = logits / (score_ms * 1e-3) / 148 / (sm_mhz * 1e6)
-    roofline = {"bound": "hbm", "kernel": "score_tc_kernel (window QK^T on tcgen05 + softmax partials), one launch per step",
+    kernel_name = ("score_fast_kernel" if args.scoring == "fast" else "score_tc_kernel") + \
+        " (window QK^T on tcgen05 + softmax partials), one launch per step"
+    roofline = {"bound": "hbm", "kernel": kernel_name,
                 "achieved": round(achieved, 1), "peak": peak, "peak_source": peak_src, "unit": "GB/s",
                 "frac": round(achieved / peak, 4),
                 # dram__bytes_read+write of this kernel on the B=1, L=8 copy of the workload (profiles/
-                # score_tc_kernel_cfg3_B1_L8.md: 1.043 x its K bytes), scaled by the K bytes of a full launch
-                "traffic": int(SCORE_TC_TRAFFIC_RATIO * ab["k_read"]) if SCORE_TC_TRAFFIC_RATIO else None,
+                # score_fast_kernel_cfg3_B1_L8.md: 1.047 x its K bytes), scaled by the K bytes of a full launch
+                "traffic": int(SCORE_TC_TRAFFIC_RATIO * ab["k_read"]) if SCORE_TC_TRAFFIC_RATIO and args.scoring == "fast" else None,
                 "algorithmic_bytes_per_launch": ab["k_read"], "ms_per_launch": round(score_ms, 4),
-                # what actually limits this kernel: one ex2 per logit on the special-function unit
-                # (16 lanes/clk/SM measured) and the issue slots around it
-                "also": {"bound": "alu", "unit": "ex2/clk/SM", "achieved": round(ex2_rate, 2), "peak": 16.0,
+                # what actually limits this kernel: one exponential per logit.  16 per clock per SM is what
+                # the special-function unit alone delivers (measured); the kernel takes 5 of every 16
+                # column pairs on the FMA pipe instead, so the fraction may pass 1
+                "also": {"bound": "alu", "unit": "exp/clk/SM", "achieved": round(ex2_rate, 2), "peak": 16.0,
                          "frac": round(ex2_rate / 16.0, 4), "at_sm_mhz": sm_mhz}}
     path = {"bytes_per_step": ab["total"], "k_read_bytes": ab["k_read"], "kv_gathered_bytes": ab["kv_gathered"],
             "achieved_gbs": round(ab["total"] / (ms_step * 1e-3) / 1e9, 1),
