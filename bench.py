@@ -175,6 +175,13 @@ def run_ours(args):
     if args.batch or args.layers:       # reduced copies of the workload, for profiler captures only
         cfg = cfg.replace(B=args.batch or cfg.B, L=args.layers or cfg.L,
                           name=f"{cfg.name}[B={args.batch or cfg.B},L={args.layers or cfg.L}]")
+    if args.units == "sentences":       # same tensors' shapes, units of 10-40 tokens
+        cfg = cfg.replace(S=(cfg.N - cfg.question_len) // 25, shot_dist="uniform", shot_lo=10, shot_hi=40,
+                          name=cfg.name + "[sentence units]")
+    elif args.units == "chunks":        # fixed chunks of 16 tokens; the remainder joins the question
+        S = (cfg.N - cfg.question_len) // 16
+        cfg = cfg.replace(S=S, shot_dist="uniform", shot_lo=16, shot_hi=16, question_len=cfg.N - 16 * S,
+                          name=cfg.name + "[16-token chunks]")
     dims = skv.make_dims(cfg.B, cfg.L, cfg.H, cfg.Hkv, cfg.d, cfg.N, cfg.W, cfg.S)
     pol = skv.make_policy(r_p=cfg.r_p)
     Q, K, V, off = wl.prefill_batch(cfg, dev)
@@ -443,6 +450,9 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override L (profiler captures of a smaller case)")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the number of decode steps")
     ap.add_argument("--decode-batch", type=int, default=0, help="override the decode batch (profiler captures)")
+    ap.add_argument("--units", default="shots", choices=["shots", "sentences", "chunks"],
+                    help="semantic units of the timed workload: the config's few-shot examples (default), sentence-sized "
+                         "units of 10-40 tokens (the document-QA adaptation), or fixed chunks of 16 tokens")
     ap.add_argument("--scoring", default="fast", choices=["fast", "exact"],
                     help="scoring kernel: the default pair (fast kernel + exact repair) or the exact kernel alone")
     ap.add_argument("--no-e2e", action="store_true")

@@ -314,3 +314,30 @@ def test_fast_scoring_out_of_range_items_are_recomputed(ctx, col):
     gpu = P.gpu_prefill(ctx, dims, Q, K, V, off, cfg.r_p, 0, "fused")
     assert skv.shotkv_repaired_items(ctx) == before
     P.check_all_units(gpu, Q, K, V, off, cfg.r_p)
+
+
+def test_sentence_sized_units_full_path(ctx):
+    """Document-QA adaptation (each sentence a semantic unit): hundreds of units of 10-40 tokens,
+    several piece ends per 128-key tile, through scoring, selection and compaction."""
+    cfg = wl.PrefillConfig("sentences", B=1, L=2, H=32, Hkv=8, d=128, N=16384, W=32, S=640, shot_dist="uniform",
+                           shot_lo=10, shot_hi=40, question_len=300, r_p=0.2, cfg_id=31)
+    for mode in (0, 1):
+        ties, gpu = run_cfg(ctx, cfg, "fused", select_mode=mode)
+        assert ties <= 2
+        assert int(gpu["kept_count"].max()) <= O.budget_tokens(cfg.r_p, cfg.N)
+
+
+def test_fixed_size_chunks_as_units(ctx):
+    """Chunk-level retention: the units are fixed-size chunks, off[i] = preamble + i*c."""
+    c, N, W, q_len, pre = 16, 8192, 64, 200, 8
+    S = (N - q_len - pre) // c
+    cfg = wl.PrefillConfig("chunks", B=2, L=1, H=32, Hkv=8, d=128, N=N, W=W, S=S, shot_dist="uniform", shot_lo=c,
+                           shot_hi=c, question_len=N - pre - S * c, preamble_len=pre, r_p=0.25, cfg_id=32)
+    Q, K, V, off = wl.prefill_batch(cfg, "cuda")
+    np.testing.assert_array_equal(off[0], pre + c * np.arange(S + 1))
+    gpu = P.gpu_prefill(ctx, P.dims_of(cfg), Q, K, V, off, cfg.r_p, 0, "fused")
+    ties = P.check_all_units(gpu, Q, K, V, off, cfg.r_p)
+    assert ties <= 2
+    kept = gpu["kept_count"].cpu().numpy()
+    always = pre + cfg.question_len
+    assert ((kept - always) % c == 0).all() and kept.max() <= O.budget_tokens(cfg.r_p, N)
