@@ -21,6 +21,9 @@ What is computed, and where the paper defines it (arXiv 2502.01941):
 * `DecodeOracle`       -- Score_decoding^l(t) = sum_h alpha_{t,h} and the TopK rule with
   k = r_d*|KV_decoding| (Sec. 5.1, decoding score and TopK equations; Algorithm 1, Phase 2), and
   KV_total = KV_prefill^C u KV_decoding^C (union equation).
+* `decode_attention`   -- the attention output o_h = sum_t alpha_{t,h} v_t over KV_total with the very
+  weights alpha_{t,h} of the decoding score equation (Preliminary: attention over the cached keys
+  and values; Sec. 5.1: the decoding score uses "the attention weight from the current step").
 
 Readings taken where the paper is silent (all listed in the design notes):
 window rows are the last W prompt positions; weights are true causal softmax
@@ -150,6 +153,24 @@ def prefill_compress(Qwin, K, V, off, r_p: float, select_mode: int = 0):
 
 
 # --------------------------------------------------------------------------- decode
+def decode_attention(q: np.ndarray, K: np.ndarray, V: np.ndarray) -> np.ndarray:
+    """o[h] = sum_t softmax_t(q_h . k_t / sqrt(d)) v_t for every query head h against its GQA
+    group's cached keys and values.  q [H, d]; K, V [Hkv, n, d] (kept prefill entries followed by
+    the decode entries, the current token included).  Returns [H, d] float64."""
+    q = np.asarray(q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    H, d = q.shape
+    G = H // K.shape[0]
+    out = np.zeros((H, d), dtype=np.float64)
+    for h in range(H):
+        g = h // G
+        s = (K[g] @ q[h]) / math.sqrt(d)
+        e = np.exp(s - s.max())
+        out[h] = (e / e.sum()) @ V[g]
+    return out
+
+
 class DecodeOracle:
     """Algorithm 1, Phase 2 for one (sequence, layer).
 
@@ -158,8 +179,13 @@ class DecodeOracle:
     step number of each entry; T = tokens generated so far.
     """
 
-    def __init__(self, Kc: np.ndarray, H: int, r_d: float, recompress_every: int):
+    def __init__(self, Kc: np.ndarray, H: int, r_d: float, recompress_every: int, Vc: np.ndarray | None = None):
+        """With `Vc` (the kept prefill values, [Hkv, M, d] as numbers) every step also computes the
+        attention output `last_out` [H, d]; `accumulate`/`step` then need `v_values`."""
         self.Kc = np.asarray(Kc, dtype=np.float64)
+        self.Vc = None if Vc is None else np.asarray(Vc, dtype=np.float64)
+        self.Vf: list[np.ndarray] = []          # decode values as numbers (only when Vc is given)
+        self.last_out = None
         self.Hkv, self.M, self.d = self.Kc.shape
         self.H = H
         self.G = H // self.Hkv
@@ -171,7 +197,7 @@ class DecodeOracle:
         self.born: list[int] = []
         self.T = 0
 
-    def accumulate(self, q: np.ndarray, k_new: np.ndarray, v_new: np.ndarray) -> None:
+    def accumulate(self, q: np.ndarray, k_new: np.ndarray, v_new: np.ndarray, v_values: np.ndarray | None = None) -> None:
         """q [H, d], k_new/v_new [Hkv, d].  Appends the new token as a decode entry with score 0,
         then adds this step's attention weights -- each head's softmax over the prefill-kept and
         decode keys together, the new token included -- to the decode entries' scores."""
@@ -192,6 +218,11 @@ class DecodeOracle:
             add += a[self.M:]
         for j in range(n):
             self.acc[j] += add[j]
+        if self.Vc is not None:
+            self.Vf.append(np.asarray(v_values, dtype=np.float64))
+            Vd = np.stack(self.Vf, axis=1)                               # [Hkv, n, d]
+            self.last_out = decode_attention(q, np.concatenate([self.Kc, Kd], axis=1),
+                                             np.concatenate([self.Vc, Vd], axis=1))
 
     def eviction_due(self) -> bool:
         return self.T % self.R == 0
@@ -214,12 +245,14 @@ class DecodeOracle:
         self.Vd = [self.Vd[j] for j in kept]
         self.acc = [self.acc[j] for j in kept]
         self.born = [self.born[j] for j in kept]
+        if self.Vc is not None:
+            self.Vf = [self.Vf[j] for j in kept]
         return evicted
 
-    def step(self, q: np.ndarray, k_new: np.ndarray, v_new: np.ndarray, decide_acc=None) -> list[int]:
+    def step(self, q: np.ndarray, k_new: np.ndarray, v_new: np.ndarray, decide_acc=None, v_values=None) -> list[int]:
         """One generation step: accumulate, then every R steps keep the top floor(r_d*T) entries.
         Returns the evicted indices (positions in the pre-eviction region)."""
-        self.accumulate(q, k_new, v_new)
+        self.accumulate(q, k_new, v_new, v_values)
         if self.eviction_due():
             return self.apply_keep(self.choose_keep(decide_acc))
         return []

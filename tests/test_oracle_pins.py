@@ -437,3 +437,71 @@ def test_pins_catch_planted_mistakes(mistake, monkeypatch):
         assert not np.allclose(bad, brute_scores(Q, K, off))
     else:
         assert not np.allclose(broken_alpha(Q, K), np.array(brute_alpha(Q, K)), atol=1e-9)
+
+
+# ---------------------------------------------------------------- decode attention output
+def _attn_inputs(H=8, Hkv=2, n=37, d=16, seed=11):
+    rng = np.random.default_rng(seed)
+    return rng.standard_normal((H, d)), rng.standard_normal((Hkv, n, d)), rng.standard_normal((Hkv, n, d))
+
+
+def test_decode_attention_matches_torch_sdpa():
+    """Pinned to a library routine the oracle does not call: torch's scaled_dot_product_attention."""
+    import torch
+    q, K, V = _attn_inputs()
+    H, Hkv = q.shape[0], K.shape[0]
+    G = H // Hkv
+    tq = torch.from_numpy(q)[:, None, :]                                  # [H, 1, d]
+    tK = torch.from_numpy(K).repeat_interleave(G, dim=0)                  # [H, n, d]
+    tV = torch.from_numpy(V).repeat_interleave(G, dim=0)
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tK, tV)[:, 0].numpy()
+    np.testing.assert_allclose(O.decode_attention(q, K, V), ref, rtol=1e-10, atol=1e-12)
+
+
+def test_decode_attention_scalar_loops_and_closed_forms():
+    q, K, V = _attn_inputs(H=4, Hkv=2, n=5, d=3, seed=3)
+    got = O.decode_attention(q, K, V)
+    for h in range(4):
+        g = h // 2
+        w = [math.exp(sum(q[h][c] * K[g][t][c] for c in range(3)) / math.sqrt(3)) for t in range(5)]
+        for c in range(3):
+            assert abs(got[h][c] - sum(w[t] * V[g][t][c] for t in range(5)) / sum(w)) < 1e-12
+    # a zero query weighs every entry alike: the output is the mean of its group's values
+    np.testing.assert_allclose(O.decode_attention(np.zeros((4, 3)), K, V), np.repeat(V.mean(axis=1), 2, axis=0), atol=1e-12)
+    # one cached entry: the output is that entry's value whatever the query
+    np.testing.assert_allclose(O.decode_attention(q, K[:, :1], V[:, :1]), np.repeat(V[:, 0], 2, axis=0), atol=1e-12)
+    # one dominant key takes all the weight
+    Kd = K.copy(); Kd[:, 2] = 0.0; Kd[0, 2] = 200.0 * q[0] / np.dot(q[0], q[0])
+    np.testing.assert_allclose(O.decode_attention(q, Kd, V)[0], V[0, 2], atol=1e-9)
+
+
+def test_decode_oracle_output_covers_prefill_and_decode_entries():
+    """The stepping oracle's `last_out` equals attention over [Vc ; decode values] including the
+    current token, and survives an eviction (values are compacted with their keys)."""
+    rng = np.random.default_rng(5)
+    H, Hkv, M, d = 4, 2, 6, 8
+    Kc, Vc = rng.standard_normal((Hkv, M, d)), rng.standard_normal((Hkv, M, d))
+    dec = O.DecodeOracle(Kc, H, r_d=0.5, recompress_every=2, Vc=Vc)
+    keys, vals = [], []
+    for s in range(6):
+        q, k, v = rng.standard_normal((H, d)), rng.standard_normal((Hkv, d)), rng.standard_normal((Hkv, d))
+        keys_before = [x.copy() for x in dec.Kd]
+        vals_before = [x.copy() for x in dec.Vf]
+        dec.step(q, k, v, v_values=v)
+        K_all = np.concatenate([Kc, np.stack(keys_before + [k], axis=1)], axis=1)
+        V_all = np.concatenate([Vc, np.stack(vals_before + [v], axis=1)], axis=1)
+        np.testing.assert_allclose(dec.last_out, O.decode_attention(q, K_all, V_all), atol=1e-12)
+        assert len(dec.Vf) == len(dec.Kd)
+        for kk, vv in zip(dec.Kd, dec.Vf):                                # pairs stay together
+            j = [i for i, x in enumerate(keys_before + [k]) if np.array_equal(x, kk)][0]
+            np.testing.assert_array_equal(vv, (vals_before + [v])[j])
+
+
+def test_decode_attention_planted_mistakes_fail():
+    q, K, V = _attn_inputs(H=4, Hkv=2, n=9, d=8, seed=8)
+    good = O.decode_attention(q, K, V)
+    wrong_group = O.decode_attention(q, K[::-1], V[::-1])
+    no_scale = O.decode_attention(q * math.sqrt(8), K, V)
+    dropped_last = O.decode_attention(q, K[:, :-1], V[:, :-1])
+    for bad in (wrong_group, no_scale, dropped_last):
+        assert np.max(np.abs(bad - good)) > 1e-3
