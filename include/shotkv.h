@@ -232,6 +232,20 @@ SHOTKV_API int shotkv_decode_step(shotkv_ctx* ctx, shotkv_decode_state* state,
                        const shotkv_bf16* q, const shotkv_bf16* k_new, const shotkv_bf16* v_new,
                        const shotkv_bf16* Kc, const int32_t* kept_count, void* stream);
 
+/* The same step with the attention output of the step fused in (Preliminary: attention over the
+ * cached keys and values; Section 5.1: the decoding score is built from "the attention weight
+ * from the current generation step", i.e. from weights a decode step computes anyway).  Besides
+ * everything shotkv_decode_step does,
+ *   attn_out[b][l][h][:] = sum_t alpha_{t,h} * v_t
+ * over the kept prefill entries (Kc, Vc rows [0, M)) and all decode entries, the new token
+ * included, with alpha the softmax weights of step 2 above; evaluated before the eviction of
+ * step 3.  K and V are each read once; the scores cost no further pass over the cache.
+ *   Vc device [B][L][Hkv][Mcap][d] bf16;  attn_out device [B][L][H][d] f32 (written in full).  */
+SHOTKV_API int shotkv_decode_step_attend(shotkv_ctx* ctx, shotkv_decode_state* state,
+                       const shotkv_bf16* q, const shotkv_bf16* k_new, const shotkv_bf16* v_new,
+                       const shotkv_bf16* Kc, const shotkv_bf16* Vc, const int32_t* kept_count,
+                       float* attn_out, void* stream);
+
 /* The work partition the scoring pass uses for `dims` on a GPU with `sm_count` SMs (host only; a
  * diagnostic and test aid).  Every prompt's keys [0, N) are cut into pieces at the shot boundaries
  * (when offsets_host is given) and at the ends of `nchunk` equal chunks of `chunk_keys` keys (whole

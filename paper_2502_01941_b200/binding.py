@@ -31,7 +31,7 @@ EXPORTS = [
     "shotkv_budget_tokens", "shotkv_kept_capacity", "shotkv_validate", "shotkv_workspace_bytes",
     "shotkv_prefill_score", "shotkv_select_shots", "shotkv_compact_kv", "shotkv_prefill_compress",
     "shotkv_host_arena_bytes", "shotkv_prefill_compress_host",
-    "shotkv_decode_workspace_bytes", "shotkv_decode_capacity", "shotkv_decode_init", "shotkv_decode_step",
+    "shotkv_decode_workspace_bytes", "shotkv_decode_capacity", "shotkv_decode_init", "shotkv_decode_step", "shotkv_decode_step_attend",
     "shotkv_profile_enable", "shotkv_profile_read", "shotkv_launch_count", "shotkv_select_shots_static", "shotkv_plan_pieces",
     "shotkv_set_scoring_mode", "shotkv_repaired_items",
 ]
@@ -93,6 +93,7 @@ def lib() -> C.CDLL:
         "shotkv_decode_capacity": (i32, [PP, i32]),
         "shotkv_decode_init": (C.c_int, [vp, PD, PP, i32, i32, vp, vp, vp, vp, vp, sz, C.POINTER(DecodeState)]),
         "shotkv_decode_step": (C.c_int, [vp, C.POINTER(DecodeState), vp, vp, vp, vp, vp, vp]),
+        "shotkv_decode_step_attend": (C.c_int, [vp, C.POINTER(DecodeState), vp, vp, vp, vp, vp, vp, vp, vp]),
         "shotkv_plan_pieces": (i32, [PD, vp, i32, C.POINTER(i32), C.POINTER(i32), vp, i32]),
         "shotkv_profile_enable": (C.c_int, [vp, C.c_int]),
         "shotkv_profile_read": (C.c_int, [vp, C.c_int, C.POINTER(C.c_float)]),
@@ -315,6 +316,18 @@ def shotkv_decode_step(ctx: Context, state: DecodeState, q, k_new, v_new, Kc, ke
                                   _ptr(v_new, device="cuda", dtype=torch.bfloat16, name="v_new"),
                                   _ptr(Kc, device="cuda", dtype=torch.bfloat16, name="Kc"),
                                   _ptr(kept_count, device="cuda", dtype=torch.int32, name="kept_count"), _stream(stream))
+    return ctx.check(rc)
+
+
+def shotkv_decode_step_attend(ctx: Context, state: DecodeState, q, k_new, v_new, Kc, Vc, kept_count, attn_out,
+                              stream=None) -> int:
+    rc = lib().shotkv_decode_step_attend(ctx._h, C.byref(state), _ptr(q, device="cuda", dtype=torch.bfloat16, name="q"),
+                                         _ptr(k_new, device="cuda", dtype=torch.bfloat16, name="k_new"),
+                                         _ptr(v_new, device="cuda", dtype=torch.bfloat16, name="v_new"),
+                                         _ptr(Kc, device="cuda", dtype=torch.bfloat16, name="Kc"),
+                                         _ptr(Vc, device="cuda", dtype=torch.bfloat16, name="Vc"),
+                                         _ptr(kept_count, device="cuda", dtype=torch.int32, name="kept_count"),
+                                         _ptr(attn_out, device="cuda", dtype=torch.float32, name="attn_out"), _stream(stream))
     return ctx.check(rc)
 
 

@@ -860,12 +860,28 @@ int shotkv_decode_init(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_po
     return SHOTKV_OK;
 }
 
-int shotkv_decode_step(shotkv_ctx* ctx, shotkv_decode_state* st, const shotkv_bf16* q, const shotkv_bf16* k_new,
-                       const shotkv_bf16* v_new, const shotkv_bf16* Kc, const int32_t* kept_count, void* stream_) {
+}  // extern "C"
+
+namespace {
+
+template <int D, int QR>
+int launch_decode_attend(shotkv_ctx* ctx, const DecodeParams& p, int U, cudaStream_t stream) {
+    const size_t smem = ((size_t)8 * p.Dcap + 8 * 8 * 2 + 16 + 8 * 17 * 8 + (size_t)8 * QR * D) * 4;
+    CUDA_TRY(ctx, cudaFuncSetAttribute(decode_attend_kernel<D, QR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    if (smem > 200 * 1024) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "Dcap too large for the attention-output step");
+    decode_attend_kernel<D, QR><<<U, 256, smem, stream>>>(p);
+    return SHOTKV_OK;
+}
+
+// One decode step; with `attn_out` the score kernel is the variant that also writes the attention output.
+int decode_step_impl(shotkv_ctx* ctx, shotkv_decode_state* st, const shotkv_bf16* q, const shotkv_bf16* k_new,
+                     const shotkv_bf16* v_new, const shotkv_bf16* Kc, const shotkv_bf16* Vc, const int32_t* kept_count,
+                     float* attn_out, void* stream_) {
     int rc = set_device(ctx);
     if (rc) return rc;
     if (!st || !q || !k_new || !v_new || !kept_count) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "pointers must not be NULL");
     if (st->Mcap > 0 && !Kc) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "Kc must not be NULL when Mcap > 0");
+    if (attn_out && st->Mcap > 0 && !Vc) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "Vc must not be NULL when Mcap > 0");
     if (st->n_dec + 1 > st->Dcap) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "decode region full: n_dec = %d, Dcap = %d", st->n_dec, st->Dcap);
     cudaStream_t stream = (cudaStream_t)stream_;
     const shotkv_dims& d = st->dims;
@@ -879,10 +895,16 @@ int shotkv_decode_step(shotkv_ctx* ctx, shotkv_decode_state* st, const shotkv_bf
     p.Kd = (__nv_bfloat16*)st->Kd; p.Vd = (__nv_bfloat16*)st->Vd; p.partial = partial;
     p.H = d.H; p.Hkv = d.Hkv; p.G = d.H / d.Hkv; p.Mcap = st->Mcap; p.Dcap = st->Dcap; p.n_old = st->n_dec;
     p.scale_log2 = kLog2e / sqrtf((float)d.d);
+    p.Vc = (const __nv_bfloat16*)Vc; p.out = attn_out;
     const size_t smem = (size_t)8 * st->Dcap * 4 + (8 * 8 * 2 + 16) * 4;
     prof_begin(ctx);
     prof_mark(ctx, stream);
-    if (d.d == 128) {
+    if (attn_out) {
+        const bool small = p.G <= 4;
+        if (d.d == 128) rc = small ? launch_decode_attend<128, 4>(ctx, p, U, stream) : launch_decode_attend<128, 8>(ctx, p, U, stream);
+        else rc = small ? launch_decode_attend<64, 4>(ctx, p, U, stream) : launch_decode_attend<64, 8>(ctx, p, U, stream);
+        if (rc) return rc;
+    } else if (d.d == 128) {
         CUDA_TRY(ctx, cudaFuncSetAttribute(decode_score_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
         decode_score_kernel<128><<<U, 256, smem, stream>>>(p);
     } else {
@@ -917,6 +939,22 @@ int shotkv_decode_step(shotkv_ctx* ctx, shotkv_decode_state* st, const shotkv_bf
     }
     prof_mark(ctx, stream);
     return SHOTKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int shotkv_decode_step(shotkv_ctx* ctx, shotkv_decode_state* st, const shotkv_bf16* q, const shotkv_bf16* k_new,
+                       const shotkv_bf16* v_new, const shotkv_bf16* Kc, const int32_t* kept_count, void* stream) {
+    return decode_step_impl(ctx, st, q, k_new, v_new, Kc, nullptr, kept_count, nullptr, stream);
+}
+
+int shotkv_decode_step_attend(shotkv_ctx* ctx, shotkv_decode_state* st, const shotkv_bf16* q, const shotkv_bf16* k_new,
+                              const shotkv_bf16* v_new, const shotkv_bf16* Kc, const shotkv_bf16* Vc,
+                              const int32_t* kept_count, float* attn_out, void* stream) {
+    if (!attn_out) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "attn_out must not be NULL");
+    return decode_step_impl(ctx, st, q, k_new, v_new, Kc, Vc, kept_count, attn_out, stream);
 }
 
 int32_t shotkv_plan_pieces(const shotkv_dims* dims, const int32_t* offsets_host, int32_t sm_count, int32_t* nchunk,

@@ -241,6 +241,13 @@ def random_prefill_cache(cfg: DecodeConfig, M: int, device="cpu", counts: np.nda
     return Kc, torch.from_numpy(np.ascontiguousarray(counts, dtype=np.int32)).to(dev)
 
 
+def random_prefill_values(cfg: DecodeConfig, M: int, device="cpu") -> torch.Tensor:
+    """The values that go with `random_prefill_cache`'s keys: Vc [B,L,Hkv,M,d] bf16 ~ N(0,1)."""
+    dev = torch.device(device)
+    g = _gen(dev, cfg.cfg_id, 405, M)
+    return torch.randn(cfg.B, cfg.L, cfg.Hkv, M, cfg.d, generator=g, device=dev).to(torch.bfloat16)
+
+
 def bf16_to_f64(x: torch.Tensor) -> np.ndarray:
     """Widen a bf16/f32 tensor to a float64 numpy array (exact)."""
     return x.detach().to("cpu", torch.float32).numpy().astype(np.float64)

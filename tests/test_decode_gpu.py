@@ -22,8 +22,10 @@ def ctx():
 
 
 class GpuDecoder:
-    def __init__(self, ctx, cfg: wl.DecodeConfig, Kc, kept_count, Dcap=None):
+    def __init__(self, ctx, cfg: wl.DecodeConfig, Kc, kept_count, Dcap=None, Vc=None):
         self.ctx, self.cfg = ctx, cfg
+        self.Vc = Vc
+        self.out = torch.zeros(cfg.B, cfg.L, cfg.H, cfg.d, dtype=torch.float32, device="cuda") if Vc is not None else None
         self.dims = skv.make_dims(cfg.B, cfg.L, cfg.H, cfg.Hkv, cfg.d, 1, 1, 0)
         self.pol = skv.make_policy(r_d=cfg.r_d, recompress_every=cfg.recompress_every)
         self.Dcap = Dcap or skv.shotkv_decode_capacity(self.pol, cfg.steps)
@@ -38,18 +40,30 @@ class GpuDecoder:
                                             self.born, self.ws)
 
     def step(self, q, k, v):
-        skv.shotkv_decode_step(self.ctx, self.state, q, k, v, self.Kc, self.kept_count)
+        if self.Vc is None:
+            skv.shotkv_decode_step(self.ctx, self.state, q, k, v, self.Kc, self.kept_count)
+        else:
+            skv.shotkv_decode_step_attend(self.ctx, self.state, q, k, v, self.Kc, self.Vc, self.kept_count, self.out)
 
 
-def lockstep(ctx, cfg, M, units, counts=None, steps=None):
+# attention outputs: |gpu - ref| <= OUT_RTOL * max|ref over the head| + OUT_ATOL.  An output is a
+# convex combination of values, so its error is measured against the head's largest component; a
+# relative test per element would be ill-posed where components cancel to nearly zero.
+OUT_RTOL, OUT_ATOL = 2e-3, 1e-6
+
+
+def lockstep(ctx, cfg, M, units, counts=None, steps=None, attend=False):
     """Runs `steps` decode steps on the GPU for the whole batch and the oracle for `units`,
-    comparing after every step.  Returns the number of reported eviction ties."""
+    comparing after every step.  With `attend` the fused attention-output step is the one run, and
+    its output is compared too.  Returns the number of reported eviction ties."""
     Kc, kept = wl.random_prefill_cache(cfg, M, "cuda", counts)
-    gpu = GpuDecoder(ctx, cfg, Kc, kept)
+    Vc = wl.random_prefill_values(cfg, M, "cuda") if attend else None
+    gpu = GpuDecoder(ctx, cfg, Kc, kept, Vc=Vc)
     orc = {}
     for (b, l) in units:
         m = int(kept[b, l])
-        orc[(b, l)] = O.DecodeOracle(wl.bf16_to_f64(Kc[b, l, :, :m]), cfg.H, cfg.r_d, cfg.recompress_every)
+        orc[(b, l)] = O.DecodeOracle(wl.bf16_to_f64(Kc[b, l, :, :m]), cfg.H, cfg.r_d, cfg.recompress_every,
+                                     Vc=wl.bf16_to_f64(Vc[b, l, :, :m]) if attend else None)
     ties = 0
     for s in range(steps or cfg.steps):
         q, k, v = wl.decode_step_inputs(cfg, s, "cuda")
@@ -59,8 +73,15 @@ def lockstep(ctx, cfg, M, units, counts=None, steps=None):
         assert gpu.state.T == s + 1
         g_born = gpu.born.cpu().numpy()
         g_acc = gpu.acc.cpu().numpy()
+        g_out = gpu.out.cpu().numpy().astype(np.float64) if attend else None
         for (b, l), o in orc.items():
-            o.accumulate(wl.bf16_to_f64(q[b, l]), wl.bf16_to_f64(k[b, l]), wl.bf16_bits(v[b, l]))
+            o.accumulate(wl.bf16_to_f64(q[b, l]), wl.bf16_to_f64(k[b, l]), wl.bf16_bits(v[b, l]),
+                         wl.bf16_to_f64(v[b, l]) if attend else None)
+            if attend:
+                ref_o = o.last_out
+                tol = OUT_RTOL * np.abs(ref_o).max(axis=1, keepdims=True) + OUT_ATOL
+                assert np.all(np.abs(g_out[b, l] - ref_o) <= tol), \
+                    f"step {s}: attention output off by {np.abs(g_out[b, l] - ref_o).max()}"
             if o.eviction_due():
                 want = o.choose_keep()
                 got_born = g_born[b, l, :n].tolist()
@@ -139,3 +160,45 @@ def test_decode_config4_shape_sampled_units(ctx):
     cfg = wl.DECODE_CONFIG
     ties = lockstep(ctx, cfg, 3276, [(0, 0), (3, 17), (7, 31)], steps=96)
     assert ties <= 3
+
+
+def test_decode_attend_small_lockstep(ctx):
+    """The fused step: scores, evictions and the attention output, G = 4 (four query rows carried)."""
+    cfg = wl.DecodeConfig("att_small", B=2, L=2, H=8, Hkv=2, d=128, steps=70, r_d=0.25, recompress_every=8, cfg_id=41)
+    counts = np.array([[100, 37], [64, 1]], np.int32)
+    assert lockstep(ctx, cfg, 100, [(0, 0), (0, 1), (1, 0), (1, 1)], counts, attend=True) <= 2
+
+
+def test_decode_attend_d64_g8_and_mha(ctx):
+    cfg = wl.DecodeConfig("att_d64", B=1, L=2, H=16, Hkv=2, d=64, steps=40, r_d=0.5, recompress_every=1, cfg_id=42)
+    assert lockstep(ctx, cfg, 33, [(0, 0), (0, 1)], attend=True) <= 2
+    cfg = wl.DecodeConfig("att_mha", B=1, L=1, H=4, Hkv=4, d=64, steps=20, r_d=1.0, recompress_every=4, cfg_id=43)
+    assert lockstep(ctx, cfg, 300, [(0, 0)], attend=True) == 0
+    cfg = wl.DecodeConfig("att_g8", B=1, L=1, H=16, Hkv=2, d=128, steps=24, r_d=0.5, recompress_every=4, cfg_id=44)
+    assert lockstep(ctx, cfg, 257, [(0, 0)], attend=True) <= 1
+
+
+def test_decode_attend_empty_prefill_region(ctx):
+    cfg = wl.DecodeConfig("att_m0", B=1, L=1, H=4, Hkv=2, d=128, steps=12, r_d=0.5, recompress_every=4, cfg_id=45)
+    assert lockstep(ctx, cfg, 8, [(0, 0)], np.zeros((1, 1), np.int32), attend=True) <= 1
+
+
+def test_decode_attend_same_scores_as_plain_step(ctx):
+    """The fused step leaves the decode state exactly as the plain step does."""
+    cfg = wl.DecodeConfig("att_same", B=2, L=1, H=8, Hkv=2, d=128, steps=20, r_d=0.25, recompress_every=4, cfg_id=46)
+    Kc, kept = wl.random_prefill_cache(cfg, 200, "cuda")
+    Vc = wl.random_prefill_values(cfg, 200, "cuda")
+    a, b = GpuDecoder(ctx, cfg, Kc, kept), GpuDecoder(ctx, cfg, Kc, kept, Vc=Vc)
+    for s in range(cfg.steps):
+        q, k, v = wl.decode_step_inputs(cfg, s, "cuda")
+        a.step(q, k, v); b.step(q, k, v)
+    torch.cuda.synchronize()
+    n = a.state.n_dec
+    assert n == b.state.n_dec and torch.equal(a.born, b.born)
+    assert torch.equal(a.Kd[:, :, :, :n], b.Kd[:, :, :, :n]) and torch.equal(a.Vd[:, :, :, :n], b.Vd[:, :, :, :n])
+    np.testing.assert_allclose(a.acc[:, :, :n].cpu().numpy(), b.acc[:, :, :n].cpu().numpy(), rtol=1e-5)
+
+
+def test_decode_attend_config4_shape_sampled_units(ctx):
+    cfg = wl.DECODE_CONFIG
+    assert lockstep(ctx, cfg, 3276, [(0, 0), (5, 9)], steps=40, attend=True) <= 2
