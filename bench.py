@@ -339,30 +339,49 @@ def decode_leg(skv, ctx, rank, world, dev, peak, args) -> dict:
     n_in = 64
     ins = [wl.decode_step_inputs(dc, s, dev) for s in range(n_in)]
 
-    def run(steps, profile=False):
+    attn_out = torch.empty(dc.B, dc.L, dc.H, dc.d, dtype=torch.float32, device=dev)
+
+    def run(steps, attend=False):
+        """`steps` decode steps from an empty decode region; returns the K bytes (and, for the
+        fused attention-output step, the V bytes as well) the score kernel had to read."""
         st = skv.shotkv_decode_init(ctx, dims, pol, Dcap, Mcap, Kd, Vd, acc, born, ws)
         bytes_read = 0
         for s in range(steps):
             q, k, v = ins[s % n_in]
-            bytes_read += (int(kept.sum()) + (st.n_dec + 1) * dc.B * dc.L) * dc.Hkv * dc.d * 2
-            skv.shotkv_decode_step(ctx, st, q, k, v, out["Kc"], out["kept_count"])
+            bytes_read += (int(kept.sum()) + (st.n_dec + 1) * dc.B * dc.L) * dc.Hkv * dc.d * 2 * (2 if attend else 1)
+            if attend:
+                skv.shotkv_decode_step_attend(ctx, st, q, k, v, out["Kc"], out["Vc"], out["kept_count"], attn_out)
+            else:
+                skv.shotkv_decode_step(ctx, st, q, k, v, out["Kc"], out["kept_count"])
         return bytes_read
 
+    def timed(steps, attend):
+        barrier(world)
+        skv.shotkv_profile_enable(ctx, True)
+        l0 = skv.shotkv_launch_count(ctx)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        nbytes = run(steps, attend)
+        e1.record()
+        barrier(world)
+        ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
+        launches = skv.shotkv_launch_count(ctx) - l0
+        st_ms = np.array([skv.shotkv_profile_read(ctx, i)[:2] for i in range(min(64, steps))])
+        skv.shotkv_profile_enable(ctx, False)
+        return ms, launches, nbytes / steps, float(st_ms[:, 0].mean())
+
     run(max(args.warmup, 3) * 8)
-    barrier(world)
-    skv.shotkv_profile_enable(ctx, True)
-    l0 = skv.shotkv_launch_count(ctx)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    bytes_read = run(dc.steps)
-    e1.record()
-    barrier(world)
-    ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
-    launches = skv.shotkv_launch_count(ctx) - l0
-    st_ms = np.array([skv.shotkv_profile_read(ctx, i)[:2] for i in range(min(64, dc.steps))])
-    skv.shotkv_profile_enable(ctx, False)
-    per_step_bytes = bytes_read / dc.steps
-    score_ms = float(st_ms[:, 0].mean())
+    ms, launches, per_step_bytes, score_ms = timed(dc.steps, False)
+    # the same steps with the attention output fused into the score kernel (K and V both read)
+    a_steps = min(dc.steps, 256)
+    run(8, True)
+    a_ms, a_launches, a_bytes, a_score_ms = timed(a_steps, True)
+    attend = {"metric": "decode steps/sec, attention output fused", "value": round(a_steps * world / (a_ms * 1e-3), 1),
+              "unit": "steps/s", "steps": a_steps, "ms_per_step": round(a_ms / a_steps, 4), "gpu_launches": int(a_launches),
+              "roofline": {"bound": "hbm", "kernel": "decode_attend_kernel (last 64 steps)",
+                           "achieved": round(a_bytes / (a_score_ms * 1e-3) / 1e9, 1), "peak": peak, "unit": "GB/s",
+                           "frac": round(a_bytes / (a_score_ms * 1e-3) / 1e9 / peak, 4), "traffic": None,
+                           "algorithmic_bytes_per_launch": int(a_bytes), "ms_per_launch": round(a_score_ms, 4)}}
     return {"metric": "decode steps/sec", "value": round(dc.steps * world / (ms * 1e-3), 1), "unit": "steps/s",
             "note": "one step = all 8 sequences x 32 layers of one replica; value sums the replicas",
             "steps": dc.steps, "ms_per_step": round(ms / dc.steps, 4), "gpu_launches": int(launches),
@@ -375,7 +394,8 @@ def decode_leg(skv, ctx, rank, world, dev, peak, args) -> dict:
                          # profiles/decode_score_kernel_cfg4_B2.md: dram read+write = 1.012 x algorithmic
                          "traffic": int(DECODE_TRAFFIC_RATIO * per_step_bytes) if DECODE_TRAFFIC_RATIO else None,
                          "algorithmic_bytes_per_launch": int(per_step_bytes), "ms_per_launch": round(score_ms, 4)},
-            "path_frac_of_measured_hbm": round(per_step_bytes / (ms / dc.steps * 1e-3) / 1e9 / peak, 4)}
+            "path_frac_of_measured_hbm": round(per_step_bytes / (ms / dc.steps * 1e-3) / 1e9 / peak, 4),
+            "attend": attend}
 
 
 # ------------------------------------------------------------------ the oracle, timed
