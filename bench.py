@@ -45,6 +45,7 @@ FALLBACK_HBM_GBS = 6650.0
 # profiles/score_fast_kernel_cfg3_B1_L8.md; set to None whenever the kernel changes after the capture.
 SCORE_TC_TRAFFIC_RATIO = 1.047
 DECODE_TRAFFIC_RATIO = 1.012    # profiles/decode_score_kernel_cfg4_B2.md
+DECODE_ATTEND_TRAFFIC_RATIO = 1.006    # profiles/decode_attend_kernel_cfg4_B2.md
 NOMINAL_HBM_GBS = 8000.0
 
 
@@ -380,7 +381,8 @@ def decode_leg(skv, ctx, rank, world, dev, peak, args) -> dict:
               "unit": "steps/s", "steps": a_steps, "ms_per_step": round(a_ms / a_steps, 4), "gpu_launches": int(a_launches),
               "roofline": {"bound": "hbm", "kernel": "decode_attend_kernel (last 64 steps)",
                            "achieved": round(a_bytes / (a_score_ms * 1e-3) / 1e9, 1), "peak": peak, "unit": "GB/s",
-                           "frac": round(a_bytes / (a_score_ms * 1e-3) / 1e9 / peak, 4), "traffic": None,
+                           "frac": round(a_bytes / (a_score_ms * 1e-3) / 1e9 / peak, 4),
+                           "traffic": int(DECODE_ATTEND_TRAFFIC_RATIO * a_bytes) if DECODE_ATTEND_TRAFFIC_RATIO else None,
                            "algorithmic_bytes_per_launch": int(a_bytes), "ms_per_launch": round(a_score_ms, 4)}}
     return {"metric": "decode steps/sec", "value": round(dc.steps * world / (ms * 1e-3), 1), "unit": "steps/s",
             "note": "one step = all 8 sequences x 32 layers of one replica; value sums the replicas",
