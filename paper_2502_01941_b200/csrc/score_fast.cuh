@@ -19,8 +19,9 @@
 //   * One ex2 per logit is the ceiling of the special-function unit (16 lanes per clock per SM),
 //     so PE of every 16 column pairs take their exponentials on the FMA pipe instead: round to nearest
 //     integer n by the magic-number addition, a cubic in the remainder f in [-1/2, 1/2]
-//     (relative error below 7.5e-5), and n added into the exponent field.  The argument is
-//     clamped to [-125, 128] first, so the result is a normal number, or +inf at the top.
+//     (relative error below 7.5e-5), and n added into the exponent field.  A saturating
+//     multiply-add clamps the argument to [-126, 128] first, so the result is a normal number,
+//     or +inf at the top.
 #pragma once
 #include "score_tc.cuh"
 
@@ -48,21 +49,28 @@ namespace tc {
 constexpr float kRefShift = 32.f;        // the first tile's row maximum is exponentiated to 2^-32
 constexpr float kRedoAbove = 1e30f;      // a partial sum at or above this sends its item to the exact kernel
 
-// 2^x on the FMA pipe for two values at a time (packed fp32 pairs), x clamped to [-125, 128].
-// The packed multiply-adds take one issue slot for two columns, which is what makes room for
-// this path beside the special-function one.
-__device__ __forceinline__ uint64_t exp2_fma2(uint64_t x2) {
-    float xa, xb;
-    unpack2(x2, xa, xb);
-    xa = fminf(fmaxf(xa, -125.f), 128.f);
-    xb = fminf(fmaxf(xb, -125.f), 128.f);
-    const uint64_t xc = pack2(xa, xb);
-    const uint64_t t = fadd2(xc, pack2(12582912.f, 12582912.f));       // 1.5 * 2^23: the low mantissa bits hold round(x)
-    const uint64_t fl = fadd2(t, pack2(-12582912.f, -12582912.f));
-    const uint64_t f = ffma2(fl, pack2(-1.f, -1.f), xc);                // in [-1/2, 1/2]
-    uint64_t q = ffma2(pack2(5.5171668e-02f, 5.5171668e-02f), f, pack2(2.4261112e-01f, 2.4261112e-01f));
-    q = ffma2(q, f, pack2(6.9326099e-01f, 6.9326099e-01f));
-    q = ffma2(q, f, pack2(9.9992807e-01f, 9.9992807e-01f));
+// 2^x on the FMA pipe for two logits at a time, x = s * scale + neg.  One saturating
+// multiply-add per logit maps x from [-126, 128] onto y in [0, 1] and so does the scaling, the
+// shift and both clamps at once (c1 = scale / 254, c0 = (neg + 126) / 254; the grid of y costs
+// x an absolute error below 8e-6).  Then, on packed pairs: t = 254 y + (1.5 * 2^23 - 126) rounds
+// to the nearest integer n = round(x) in its low mantissa bits, t - (1.5 * 2^23 - 126) = n + 126
+// exactly, g = (n + 126) - 254 y = -(x - n) lies in [-1/2, 1/2], a cubic in g gives 2^(x - n)
+// (relative error below 7.5e-5) and n is added into the exponent field.  x >= 128 yields +inf,
+// x <= -126 a number below 2^-125; nothing in between leaves the normal range.
+__device__ __forceinline__ float fma_sat(float a, float b, float c) {
+    float d;
+    asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t exp2_fma2(float sa, float sb, float c1, float c0) {
+    constexpr float kMagic = 12582912.f - 126.f;
+    const uint64_t y = pack2(fma_sat(sa, c1, c0), fma_sat(sb, c1, c0));
+    const uint64_t t = ffma2(y, pack2(254.f, 254.f), pack2(kMagic, kMagic));
+    const uint64_t fl = fadd2(t, pack2(-kMagic, -kMagic));
+    const uint64_t g = ffma2(y, pack2(-254.f, -254.f), fl);
+    uint64_t q = ffma2(pack2(-5.5171668e-02f, -5.5171668e-02f), g, pack2(2.4261112e-01f, 2.4261112e-01f));
+    q = ffma2(q, g, pack2(-6.9326099e-01f, -6.9326099e-01f));
+    q = ffma2(q, g, pack2(9.9992807e-01f, 9.9992807e-01f));
     float qa, qb, ta, tb;
     unpack2(q, qa, qb);
     unpack2(t, ta, tb);
@@ -78,9 +86,9 @@ __device__ __forceinline__ constexpr bool pair_on_fma(int j) {
 
 // 2^(r[i] * scale + neg) for the column pair (2j, 2j+1), packed
 template <int NP>
-__device__ __forceinline__ uint64_t exp_pair(const uint32_t (&r)[32], int j, uint64_t sc2, uint64_t ng2) {
+__device__ __forceinline__ uint64_t exp_pair(const uint32_t (&r)[32], int j, uint64_t sc2, uint64_t ng2, float c1, float c0) {
+    if (pair_on_fma<NP>(j)) return exp2_fma2(SKV_F(r, 2 * j), SKV_F(r, 2 * j + 1), c1, c0);
     const uint64_t x2 = ffma2(pack2(SKV_F(r, 2 * j), SKV_F(r, 2 * j + 1)), sc2, ng2);
-    if (pair_on_fma<NP>(j)) return exp2_fma2(x2);
     float xa, xb;
     unpack2(x2, xa, xb);
     return pack2(ex2f(xa), ex2f(xb));
@@ -90,18 +98,20 @@ __device__ __forceinline__ uint64_t exp_pair(const uint32_t (&r)[32], int j, uin
 template <int NP>
 __device__ __forceinline__ void expacc32(const uint32_t (&r)[32], float scale, float neg, uint64_t (&z)[2]) {
     const uint64_t sc2 = pack2(scale, scale), ng2 = pack2(neg, neg);
+    const float c1 = scale * (1.f / 254.f), c0 = (neg + 126.f) * (1.f / 254.f);
 #pragma unroll
-    for (int j = 0; j < 16; ++j) z[j & 1] = fadd2(z[j & 1], exp_pair<NP>(r, j, sc2, ng2));
+    for (int j = 0; j < 16; ++j) z[j & 1] = fadd2(z[j & 1], exp_pair<NP>(r, j, sc2, ng2, c1, c0));
 }
 
 // r[i] = 2^(r[i] * scale + neg) in place, the same split between the two pipes
 template <int NP>
 __device__ __forceinline__ void exp32_mixed(uint32_t (&r)[32], float scale, float neg) {
     const uint64_t sc2 = pack2(scale, scale), ng2 = pack2(neg, neg);
+    const float c1 = scale * (1.f / 254.f), c0 = (neg + 126.f) * (1.f / 254.f);
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
         float ea, eb;
-        unpack2(exp_pair<NP>(r, j, sc2, ng2), ea, eb);
+        unpack2(exp_pair<NP>(r, j, sc2, ng2, c1, c0), ea, eb);
         r[2 * j] = __float_as_uint(ea);
         r[2 * j + 1] = __float_as_uint(eb);
     }
