@@ -290,8 +290,13 @@ def e2e_leg(skv, ctx, cfg, dims, pol, Q, K, V, off, Mcap, world, dev, args) -> d
         arena = torch.empty(skv.shotkv_host_arena_bytes(dims, Mcap), dtype=torch.uint8, device=dev)
     except RuntimeError as e:
         return {"value": None, "unit": UNIT, "error": f"could not allocate pinned host buffers: {str(e)[:100]}"}
-    h2d = sum(t.numel() * t.element_size() for t in (hQ, hK, hV))
-    d2h = sum(ho[k].numel() * ho[k].element_size() for k in ("shot_scores", "keep", "kept_idx", "kept_count", "Kc", "Vc"))
+    # bytes that cross the bus per step: Q and K are copied whole; of V only the kept tokens' rows are
+    # read (the compaction kernel gathers them from the page-locked host tensor); Kc and Vc rows are
+    # written to the page-locked host outputs by that kernel; the small result arrays are copied
+    row_bytes = cfg.d * 2
+    kept_rows = None            # filled in after the first step, from its own kept counts
+    h2d_fixed = sum(t.numel() * t.element_size() for t in (hQ, hK))
+    d2h_fixed = sum(ho[k].numel() * ho[k].element_size() for k in ("shot_scores", "keep", "kept_idx", "kept_count"))
 
     def step():
         skv.shotkv_prefill_compress_host(ctx, dims, pol, hQ, hK, hV, off, ho["shot_scores"], ho["keep"], ho["kept_idx"],
@@ -299,6 +304,9 @@ def e2e_leg(skv, ctx, cfg, dims, pol, Q, K, V, off, Mcap, world, dev, args) -> d
     steps = max(2, min(args.steps, args.e2e_steps))
     step()
     barrier(world)
+    kept_rows = int(ho["kept_count"].to(torch.int64).sum()) * cfg.Hkv
+    h2d = h2d_fixed + kept_rows * row_bytes
+    d2h = d2h_fixed + 2 * kept_rows * row_bytes
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(steps):
@@ -308,7 +316,8 @@ def e2e_leg(skv, ctx, cfg, dims, pol, Q, K, V, off, Mcap, world, dev, args) -> d
     ms = max_over_ranks(e0.elapsed_time(e1), world, dev) / steps
     return {"value": round(cfg.B * cfg.N * world / (ms * 1e-3), 1), "unit": UNIT, "ms_per_step": round(ms, 3),
             "steps": steps, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-            "api": "shotkv_prefill_compress_host"}
+            "api": "shotkv_prefill_compress_host",
+            "note": "page-locked host tensors: Q and K copied whole, V rows of kept tokens gathered in place, Kc/Vc written in place"}
 
 
 def decode_leg(skv, ctx, rank, world, dev, peak, args) -> dict:

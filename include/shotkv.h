@@ -176,9 +176,14 @@ SHOTKV_API int shotkv_prefill_compress(shotkv_ctx* ctx, const shotkv_dims* dims,
                             float* token_importance, uint32_t flags,
                             void* ws, size_t ws_bytes, void* stream);
 
-/* Same, for callers whose tensors live in HOST memory (pinned memory makes the copies
- * asynchronous).  Copies Qwin/K/V to the device arena, runs Phase 1, copies the results back, all
- * on `stream`; returns after enqueueing.  Outputs with a NULL host pointer are not copied back.
+/* Same, for callers whose tensors live in HOST memory.  Copies Qwin and K to the device arena, runs
+ * Phase 1 and delivers the results to the host buffers, all on `stream`; returns after
+ * enqueueing.  Outputs with a NULL host pointer are not delivered.
+ *   Page-locked buffers (cudaHostAlloc / cudaHostRegister) make the copies asynchronous, and
+ *   more: V is only ever gathered (the Compress equation takes the kept tokens' rows), so a
+ *   page-locked V_host is read in place by the compaction kernel -- only the kept rows cross the
+ *   bus -- and page-locked Kc_host / Vc_host are written in place by it (rows at and beyond
+ *   kept_count are then left untouched).  Pageable buffers are staged whole through the arena.
  *   arena  device buffer of >= shotkv_host_arena_bytes(dims, Mcap) bytes, 256-byte aligned
  * The host outputs are valid once `stream` has been synchronised.  */
 SHOTKV_API size_t shotkv_host_arena_bytes(const shotkv_dims* dims, int32_t Mcap);

@@ -794,19 +794,40 @@ int shotkv_prefill_compress_host(shotkv_ctx* ctx, const shotkv_dims* dims, const
     if (arena_bytes < a.total) return fail(ctx, SHOTKV_ERR_WORKSPACE_TOO_SMALL, "arena has %zu bytes, %zu needed", arena_bytes, a.total);
     cudaStream_t stream = (cudaStream_t)stream_;
     const size_t BL = (size_t)dims->B * dims->L, U = BL * dims->Hkv;
+    // Page-locked host buffers are addressable from the device.  V is only ever gathered (the rows
+    // of the kept tokens), so a page-locked V is read in place by the compaction kernel instead of
+    // being copied whole, and page-locked Kc/Vc are written in place by it.  Pageable buffers take
+    // the staged copies through the arena.
+    auto device_alias = [](const void* host) -> void* {
+        if (!host) return nullptr;
+        cudaPointerAttributes at{};
+        if (cudaPointerGetAttributes(&at, host) != cudaSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+    };
+    const shotkv_bf16* V_in = (const shotkv_bf16*)device_alias(V_host);
+    shotkv_bf16* Kc_out = (shotkv_bf16*)device_alias(Kc_host);
+    shotkv_bf16* Vc_out = (shotkv_bf16*)device_alias(Vc_host);
+    if (((uintptr_t)V_in | (uintptr_t)Kc_out | (uintptr_t)Vc_out) & 15) V_in = nullptr, Kc_out = Vc_out = nullptr;
     CUDA_TRY(ctx, cudaMemcpyAsync(a.Q, Qwin_host, BL * dims->H * dims->W * dims->d * 2, cudaMemcpyHostToDevice, stream));
     CUDA_TRY(ctx, cudaMemcpyAsync(a.K, K_host, U * dims->N * dims->d * 2, cudaMemcpyHostToDevice, stream));
-    CUDA_TRY(ctx, cudaMemcpyAsync(a.V, V_host, U * dims->N * dims->d * 2, cudaMemcpyHostToDevice, stream));
-    const int prc = shotkv_prefill_compress(ctx, dims, policy, a.Q, a.K, a.V, offsets_host, a.scores, a.keep, a.idx, a.count,
-                                            Mcap, a.Kc, a.Vc, nullptr, 0, a.ws, a.ws_bytes, stream_);
+    if (!V_in) {
+        CUDA_TRY(ctx, cudaMemcpyAsync(a.V, V_host, U * dims->N * dims->d * 2, cudaMemcpyHostToDevice, stream));
+        V_in = a.V;
+    }
+    const int prc = shotkv_prefill_compress(ctx, dims, policy, a.Q, a.K, V_in, offsets_host, a.scores, a.keep, a.idx, a.count,
+                                            Mcap, Kc_out ? Kc_out : a.Kc, Vc_out ? Vc_out : a.Vc, nullptr, 0, a.ws,
+                                            a.ws_bytes, stream_);
     if (prc < 0) return prc;
     const size_t S1 = dims->S > 0 ? dims->S : 1;
     if (shot_scores_host) CUDA_TRY(ctx, cudaMemcpyAsync(shot_scores_host, a.scores, BL * S1 * 4, cudaMemcpyDeviceToHost, stream));
     if (keep_host) CUDA_TRY(ctx, cudaMemcpyAsync(keep_host, a.keep, BL * S1, cudaMemcpyDeviceToHost, stream));
     if (kept_idx_host) CUDA_TRY(ctx, cudaMemcpyAsync(kept_idx_host, a.idx, BL * (size_t)Mcap * 4, cudaMemcpyDeviceToHost, stream));
     if (kept_count_host) CUDA_TRY(ctx, cudaMemcpyAsync(kept_count_host, a.count, BL * 4, cudaMemcpyDeviceToHost, stream));
-    if (Kc_host) CUDA_TRY(ctx, cudaMemcpyAsync(Kc_host, a.Kc, U * (size_t)Mcap * dims->d * 2, cudaMemcpyDeviceToHost, stream));
-    if (Vc_host) CUDA_TRY(ctx, cudaMemcpyAsync(Vc_host, a.Vc, U * (size_t)Mcap * dims->d * 2, cudaMemcpyDeviceToHost, stream));
+    if (Kc_host && !Kc_out) CUDA_TRY(ctx, cudaMemcpyAsync(Kc_host, a.Kc, U * (size_t)Mcap * dims->d * 2, cudaMemcpyDeviceToHost, stream));
+    if (Vc_host && !Vc_out) CUDA_TRY(ctx, cudaMemcpyAsync(Vc_host, a.Vc, U * (size_t)Mcap * dims->d * 2, cudaMemcpyDeviceToHost, stream));
     return prc;
 }
 

@@ -222,6 +222,23 @@ def test_host_buffer_entry_point(ctx):
     P.check_all_units(hout, Q, K, V, off, cfg.r_p)
 
 
+def test_host_buffer_entry_point_pageable_memory(ctx):
+    """Pageable host buffers cannot be addressed from the device: everything is staged through the arena."""
+    cfg = SHRUNK[3]
+    Q, K, V, off = wl.prefill_batch(cfg, "cpu")
+    dims = P.dims_of(cfg)
+    pol = skv.make_policy(r_p=cfg.r_p)
+    Mcap = skv.shotkv_kept_capacity(dims, pol, off)
+    hout = skv.alloc_prefill_outputs(dims, Mcap, device="cpu")
+    assert not K.is_pinned() and not hout["Kc"].is_pinned()
+    arena = torch.empty(skv.shotkv_host_arena_bytes(dims, Mcap), dtype=torch.uint8, device="cuda")
+    skv.shotkv_prefill_compress_host(ctx, dims, pol, Q, K, V, off, hout["shot_scores"], hout["keep"], hout["kept_idx"],
+                                     hout["kept_count"], Mcap, hout["Kc"], hout["Vc"], arena)
+    torch.cuda.synchronize()
+    hout["token_importance"] = None
+    P.check_all_units(hout, Q, K, V, off, cfg.r_p)
+
+
 def test_errors_are_reported_not_computed(ctx):
     cfg = wl.CONFIGS[0]
     Q, K, V, off = wl.prefill_batch(cfg, "cuda")
