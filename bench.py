@@ -257,6 +257,28 @@ def run_ours(args):
         "roofline": roofline, "path": path, "clocks": clocks, "gpu_launches": int(launches),
     }
 
+    # ---------------- the per-token form of the step (shotkv_prefill_score: a second pass over K
+    # that normalises and column-sums, then selection from token importances, then compaction)
+    if not args.no_tokens:
+        imp = torch.empty(cfg.B, cfg.L, cfg.Hkv, cfg.N, dtype=torch.float32, device=dev)
+        def tok_step():
+            skv.shotkv_prefill_compress(ctx, dims, pol, Q, K, V, off, out["shot_scores"], out["keep"], out["kept_idx"],
+                                        out["kept_count"], Mcap, out["Kc"], out["Vc"], imp, skv.FLAG_TOKEN_IMPORTANCE, out["ws"])
+        tok_step()
+        barrier(world)
+        n_tok = max(2, min(args.steps, 10))
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(n_tok):
+            tok_step()
+        t1.record()
+        barrier(world)
+        tok_ms = max_over_ranks(t0.elapsed_time(t1), world, dev) / n_tok
+        result["token_importance_path"] = {
+            "value": round(tokens / (tok_ms * 1e-3), 1), "unit": UNIT, "ms_per_step": round(tok_ms, 4), "steps": n_tok,
+            "note": "same step with SHOTKV_FLAG_TOKEN_IMPORTANCE: per-token importance materialised (two passes over K)",
+            "frac_of_measured_hbm_for_two_k_reads": round((ab["total"] + ab["k_read"]) / (tok_ms * 1e-3) / 1e9 / peak, 4)}
+        del imp
     # ---------------- end to end from host buffers (rank-local, same workload)
     if not args.no_e2e:
         result["e2e"] = e2e_leg(skv, ctx, cfg, dims, pol, Q, K, V, off, Mcap, world, dev, args)
@@ -486,6 +508,7 @@ def main():
                          "units of 10-40 tokens (the document-QA adaptation), or fixed chunks of 16 tokens")
     ap.add_argument("--scoring", default="fast", choices=["fast", "exact"],
                     help="scoring kernel: the default pair (fast kernel + exact repair) or the exact kernel alone")
+    ap.add_argument("--no-tokens", action="store_true", help="skip the per-token-importance form of the step")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")

@@ -137,7 +137,7 @@ __global__ void __launch_bounds__(ScoreFastCfg<D, MB>::kThreads, 1)
     const int item_end = (int)(total * (blockIdx.x + 1) / gridDim.x);
 
     if (warp == 0) {
-        if (lane == 0) tc::producer_role<D, MB, false>(pp, &tmQ, &tmK, q_box_rows, k_box_rows, p, item_begin, item_end);
+        if (lane == 0) tc::producer_role<D, MB, false, false>(pp, &tmQ, &tmK, q_box_rows, k_box_rows, p, item_begin, item_end);
     } else if (warp == 1 || warp == 2) {
         if (lane == 0) tc::mma_role<D, MB, false, 2>(pp, p, item_begin, item_end, warp - 1);
     } else if (warp >= 4) {

@@ -16,7 +16,7 @@
 //               a chunk.  The slices of a row are merged through shared memory when a piece is
 //               complete, in a fixed order.
 // The reductions over pieces, rows and heads that turn (m, z) into shot scores are done by the
-// kernels in score_mma.cuh.
+// kernels in reductions.cuh.
 //
 // Every wait on an mbarrier is bounded: after about two seconds a waiter raises the CTA's abort
 // flag and the device error word, all roles leave their loops, outstanding bulk copies are
@@ -376,7 +376,9 @@ __device__ __forceinline__ float* pipe_scratch(const Pipe<Cfg>& pp, unsigned cha
 
 // One thread: the unit's window queries (once per unit) and K tiles of 128 keys into the ring.
 // FILTERED: skip the items whose redo flag is clear (the exact kernel's repair launches).
-template <int D, int MB, bool FILTERED, class Cfg>
+// QKMAJOR: lay Q out k-block major (all rows of one 64-element k block contiguous), as a B
+// operand of more than 128 rows needs; otherwise row-block major (each 128-row block contiguous).
+template <int D, int MB, bool FILTERED, bool QKMAJOR, class Cfg>
 __device__ __forceinline__ void producer_role(const Pipe<Cfg>& pp, const CUtensorMap* tmQ, const CUtensorMap* tmK,
                                               int q_box_rows, int k_box_rows, const ScoreTcParams& p, int item_begin,
                                               int item_end) {
@@ -398,7 +400,8 @@ __device__ __forceinline__ void producer_role(const Pipe<Cfg>& pp, const CUtenso
             for (int b = 0; b < MB; ++b)
 #pragma unroll
                 for (int sub = 0; sub < NSUB; ++sub)
-                    tma_load_2d(pp.sQ + (b * NSUB + sub) * Cfg::kSubBytes, tmQ, sub * 64, u * p.R + b * 128, pp.qfull());
+                    tma_load_2d(pp.sQ + (QKMAJOR ? sub * MB + b : b * NSUB + sub) * Cfg::kSubBytes, tmQ, sub * 64, u * p.R + b * 128,
+                                pp.qfull());
             cur_u = u;
         }
         for (int t = 0; t < nt; ++t) {
@@ -514,7 +517,7 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
     const int item_end = (int)(total * (blockIdx.x + 1) / gridDim.x);
 
     if (warp == 0) {
-        if (lane == 0) tc::producer_role<D, MB, true>(pp, &tmQ, &tmK, q_box_rows, k_box_rows, p, item_begin, item_end);
+        if (lane == 0) tc::producer_role<D, MB, true, false>(pp, &tmQ, &tmK, q_box_rows, k_box_rows, p, item_begin, item_end);
     } else if (warp == 1) {
         if (lane == 0) tc::mma_role<D, MB, true, 1>(pp, p, item_begin, item_end, 0);
     } else if (warp >= 4) {

@@ -12,10 +12,11 @@
 #include <new>
 #include <vector>
 
+#include "colsum_tc.cuh"
 #include "common.cuh"
 #include "decode.cuh"
 #include "score_fast.cuh"
-#include "score_mma.cuh"
+#include "reductions.cuh"
 #include "score_tc.cuh"
 #include "select_compact.cuh"
 
@@ -263,39 +264,6 @@ int build_pieces(const shotkv_dims* d, const int32_t* off, const ChunkPlan& plan
     return (int)P;
 }
 
-template <int D, int MB>
-int launch_colsum_t(shotkv_ctx* ctx, const ScoreParams& sp, int U, cudaStream_t stream) {
-    constexpr int smem = score_mma_smem_bytes<D, MB>();
-    CUDA_TRY(ctx, cudaFuncSetAttribute(column_sum_mma_kernel<D, MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    dim3 grid((sp.P + sp.ppc - 1) / sp.ppc, U);
-    column_sum_mma_kernel<D, MB><<<grid, 256, smem, stream>>>(sp);
-    LAUNCH_CHECK(ctx);
-    return SHOTKV_OK;
-}
-
-int launch_colsum(shotkv_ctx* ctx, const shotkv_dims* d, const ScoreParams& sp, int U, cudaStream_t stream) {
-    const bool big = sp.Rpad == 256;
-    if (d->d == 128) return big ? launch_colsum_t<128, 2>(ctx, sp, U, stream) : launch_colsum_t<128, 1>(ctx, sp, U, stream);
-    return big ? launch_colsum_t<64, 2>(ctx, sp, U, stream) : launch_colsum_t<64, 1>(ctx, sp, U, stream);
-}
-
-ScoreParams base_params(const shotkv_dims* d, const shotkv_bf16* Q, const shotkv_bf16* K, const PrefillWs& w, int P) {
-    ScoreParams sp{};
-    sp.Q = reinterpret_cast<const __nv_bfloat16*>(Q);
-    sp.K = reinterpret_cast<const __nv_bfloat16*>(K);
-    sp.pieces = w.pieces;
-    sp.P = P;
-    const long long U = (long long)d->B * d->L * d->Hkv;
-    int ppc = (int)((U * P) / (148 * 8));     // aim for >= 8 work items per SM
-    sp.ppc = ppc < 1 ? 1 : (ppc > 8 ? 8 : ppc);
-    sp.L = d->L; sp.H = d->H; sp.Hkv = d->Hkv; sp.N = d->N; sp.W = d->W;
-    sp.G = d->H / d->Hkv; sp.R = sp.G * d->W; sp.Rpad = rpad_of(d);
-    sp.scale_log2 = kLog2e / sqrtf((float)d->d);
-    sp.row_m = w.row_m; sp.row_invz = w.row_invz;
-    sp.imp = nullptr;
-    return sp;
-}
-
 int set_device(shotkv_ctx* ctx) {
     if (!ctx) return SHOTKV_ERR_INVALID_ARG;
     CUDA_TRY(ctx, cudaSetDevice(ctx->device));
@@ -350,33 +318,41 @@ int launch_score_fast_t(shotkv_ctx* ctx, const CUtensorMap& tmQ, const CUtensorM
     return SHOTKV_OK;
 }
 
-int launch_score_tc(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const shotkv_bf16* K, const PrefillWs& w,
-                    int P, const ChunkPlan& plan, cudaStream_t stream) {
+// Tensor maps of Q (2-D: d x rows) and K (3-D: d x N x units), 64-element boxes with 128-byte swizzle, and the
+// parameters every tensor-core pass shares.
+struct TcSetup {
+    CUtensorMap tmQ, tmK;
+    int qbox, kbox;
+    ScoreTcParams sp;
+};
+int tc_setup(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const shotkv_bf16* K, const PrefillWs& w, int P,
+             const ChunkPlan& plan, TcSetup& t) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return fail(ctx, SHOTKV_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
     if (((uintptr_t)Q | (uintptr_t)K) & 15) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "Qwin and K must be 16-byte aligned");
     const long long U = (long long)d->B * d->L * d->Hkv;
     const int R = (d->H / d->Hkv) * d->W;
     const long long qrows = U * R;
-    const int qbox = qrows < 128 ? (int)qrows : 128, kbox = d->N < 128 ? d->N : 128;
-    CUtensorMap tmQ, tmK;
+    t.qbox = qrows < 128 ? (int)qrows : 128;
+    t.kbox = d->N < 128 ? d->N : 128;
     {
         cuuint64_t dims[2] = {(cuuint64_t)d->d, (cuuint64_t)qrows};
         cuuint64_t strides[1] = {(cuuint64_t)d->d * 2};
-        cuuint32_t box[2] = {64, (cuuint32_t)qbox}, es[2] = {1, 1};
-        CUresult r = enc(&tmQ, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)Q, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+        cuuint32_t box[2] = {64, (cuuint32_t)t.qbox}, es[2] = {1, 1};
+        CUresult r = enc(&t.tmQ, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)Q, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return fail(ctx, SHOTKV_ERR_CUDA, "cuTensorMapEncodeTiled(Qwin) failed with %d", (int)r);
     }
     {
         cuuint64_t dims[3] = {(cuuint64_t)d->d, (cuuint64_t)d->N, (cuuint64_t)U};
         cuuint64_t strides[2] = {(cuuint64_t)d->d * 2, (cuuint64_t)d->N * d->d * 2};
-        cuuint32_t box[3] = {64, (cuuint32_t)kbox, 1}, es[3] = {1, 1, 1};
-        CUresult r = enc(&tmK, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)K, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+        cuuint32_t box[3] = {64, (cuuint32_t)t.kbox, 1}, es[3] = {1, 1, 1};
+        CUresult r = enc(&t.tmK, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)K, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return fail(ctx, SHOTKV_ERR_CUDA, "cuTensorMapEncodeTiled(K) failed with %d", (int)r);
     }
-    ScoreTcParams sp{};
+    ScoreTcParams& sp = t.sp;
+    sp = ScoreTcParams{};
     sp.pieces = w.pieces;
     sp.chunk_first = w.chunk_first;
     sp.cf_stride = kMaxChunks + 1;
@@ -390,6 +366,44 @@ int launch_score_tc(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q,
     sp.part_m = w.part_m; sp.part_z = w.part_z;
     sp.err = ctx->err_dev;
     sp.repaired = ctx->err_dev + 1;
+    return SHOTKV_OK;
+}
+
+template <int D, int MB>
+int launch_colsum_tc_t(shotkv_ctx* ctx, const TcSetup& t, const ColsumTcParams& cp, cudaStream_t stream) {
+    constexpr int smem = ColsumTcCfg<D, MB>::kSmemBytes;
+    CUDA_TRY(ctx, cudaFuncSetAttribute(colsum_tc_kernel<D, MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    int grid = cp.base.total_items < ctx->sm_count ? cp.base.total_items : ctx->sm_count;
+    if (grid < 1) grid = 1;
+    colsum_tc_kernel<D, MB><<<grid, ColsumTcCfg<D, MB>::kThreads, smem, stream>>>(t.tmQ, t.tmK, t.qbox, t.kbox, cp);
+    LAUNCH_CHECK(ctx);
+    return SHOTKV_OK;
+}
+
+// Second pass of the per-token path: token_importance from the row statistics in the workspace.
+int launch_colsum_tc(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const shotkv_bf16* K, const PrefillWs& w,
+                     float* imp, cudaStream_t stream) {
+    TcSetup t;
+    const ChunkPlan plan = plan_chunks(d, ctx->sm_count);
+    int rc = tc_setup(ctx, d, Q, K, w, 0, plan, t);
+    if (rc) return rc;
+    ColsumTcParams cp{};
+    cp.base = t.sp;
+    cp.row_m = w.row_m; cp.row_invz = w.row_invz; cp.imp = imp;
+    const bool big = t.sp.Rpad == 256;
+    if (d->d == 128) return big ? launch_colsum_tc_t<128, 2>(ctx, t, cp, stream) : launch_colsum_tc_t<128, 1>(ctx, t, cp, stream);
+    return big ? launch_colsum_tc_t<64, 2>(ctx, t, cp, stream) : launch_colsum_tc_t<64, 1>(ctx, t, cp, stream);
+}
+
+int launch_score_tc(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const shotkv_bf16* K, const PrefillWs& w,
+                    int P, const ChunkPlan& plan, cudaStream_t stream) {
+    TcSetup t;
+    int rc0 = tc_setup(ctx, d, Q, K, w, P, plan, t);
+    if (rc0) return rc0;
+    const CUtensorMap& tmQ = t.tmQ;
+    const CUtensorMap& tmK = t.tmK;
+    const int qbox = t.qbox, kbox = t.kbox;
+    ScoreTcParams& sp = t.sp;
     const bool big = sp.Rpad == 256;
     int rc = SHOTKV_OK;
     if (ctx->scoring_mode == SHOTKV_SCORING_FAST) {
@@ -430,13 +444,12 @@ int run_stats(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const
     rc = upload_small(ctx, w.chunk_first, chunk_first.data(), chunk_first.size() * sizeof(int), stream);
     if (rc) return rc;
     const int U = d->B * d->L * d->Hkv;
-    ScoreParams sp = base_params(d, Q, K, w, P);
     prof_mark(ctx, stream);
     rc = launch_score_tc(ctx, d, Q, K, w, P, plan, stream);
     if (rc) return rc;
     prof_mark(ctx, stream);
     if (need_rows) {
-        row_stats_kernel<<<U, 256, 0, stream>>>(w.part_m, w.part_z, w.piece_seg, d->L * d->Hkv, d->S + 1, P, sp.R, sp.Rpad,
+        row_stats_kernel<<<U, 256, 0, stream>>>(w.part_m, w.part_z, w.piece_seg, d->L * d->Hkv, d->S + 1, P, (d->H / d->Hkv) * d->W, rpad_of(d),
                                                 w.row_m, w.row_invz);
         LAUNCH_CHECK(ctx);
     }
@@ -581,9 +594,7 @@ int shotkv_prefill_score(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_
     const PrefillWs w = carve(dims, ws);
     int P = 0;
     if ((rc = run_stats(ctx, dims, Qwin, K, w, nullptr, true, &P, stream))) return rc;
-    ScoreParams sp = base_params(dims, Qwin, K, w, P);
-    sp.imp = token_importance;
-    return launch_colsum(ctx, dims, sp, dims->B * dims->L * dims->Hkv, stream);
+    return launch_colsum_tc(ctx, dims, Qwin, K, w, token_importance, stream);
 }
 
 int shotkv_select_shots(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_policy* policy,
