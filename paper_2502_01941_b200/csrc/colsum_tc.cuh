@@ -14,7 +14,7 @@
 // broadcast reads.  The second group hands its partial sums to the first through a two-slot
 // shared-memory ring guarded by mbarriers; the first adds them in a fixed order and stores.
 #pragma once
-#include "score_tc.cuh"
+#include "score_fast.cuh"
 
 namespace shotkv {
 
@@ -94,7 +94,7 @@ __device__ __forceinline__ void mma_role_transposed(const Pipe<Cfg>& pp, const S
 
 }  // namespace tc
 
-template <int D, int MB>
+template <int D, int MB, int PE>
 __global__ void __launch_bounds__(ColsumTcCfg<D, MB>::kThreads, 1)
     colsum_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const int q_box_rows,
                      const int k_box_rows, const ColsumTcParams cp) {
@@ -142,8 +142,14 @@ __global__ void __launch_bounds__(ColsumTcCfg<D, MB>::kThreads, 1)
                     const float m = live ? cp.row_m[(size_t)u * p.Rpad + r] : 0.f;
                     const float iz = live ? cp.row_invz[(size_t)u * p.Rpad + r] : 0.f;
                     float* c4 = reinterpret_cast<float*>(cu + (rr >> 1));
-                    c4[rr & 1] = (live && iz > 0.f) ? -m : SHOTKV_NEG_INF;     // a row without weight exponentiates to 0
-                    c4[2 + (rr & 1)] = iz;
+                    // first two components: the additive constant of the row's exponential, -M_r where the
+                    // column pair goes to the special-function unit, (126 - M_r) / 254 where it goes to the
+                    // FMA pipe (see exp2_fma2); a row without weight gets 1/Z = 0 and a constant that exponentiates to
+                    // (nearly) zero, so that no infinity meets that zero
+                    const bool has = live && iz > 0.f;
+                    c4[rr & 1] = tc::pair_on_fma<PE>((rr >> 1) & 15) ? (has ? (126.f - m) * (1.f / 254.f) : -4.f)
+                                                                     : (has ? -m : SHOTKV_NEG_INF);
+                    c4[2 + (rr & 1)] = has ? iz : 0.f;
                     pl[rr] = live ? p.N - p.W + (r % p.W) : -1;
                 }
                 __syncwarp();
@@ -171,18 +177,26 @@ __global__ void __launch_bounds__(ColsumTcCfg<D, MB>::kThreads, 1)
                         __syncwarp();
                         if (lane == 0) tc::mbar_arrive(pp.tempty(acc, 0));
                     }
-                    if (!plain) {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (key > pl[c * 32 + i]) r[i] = 0xff800000u;   // after the row's own position: no weight
-                    }
+                    const float c1 = scale * (1.f / 254.f);
 #pragma unroll
                     for (int jp = 0; jp < 16; ++jp) {
                         const float4 k4 = cu[c * 16 + jp];
-                        const uint64_t x2 = tc::ffma2(tc::pack2(SKV_F(r, 2 * jp), SKV_F(r, 2 * jp + 1)), sc2, tc::pack2(k4.x, k4.y));
-                        float xa, xb;
-                        tc::unpack2(x2, xa, xb);
-                        s2[jp & 1] = tc::ffma2(tc::pack2(ex2f(xa), ex2f(xb)), tc::pack2(k4.z, k4.w), s2[jp & 1]);
+                        uint64_t e2;
+                        if (tc::pair_on_fma<PE>(jp)) {
+                            const float2 y = make_float2(tc::fma_sat(SKV_F(r, 2 * jp), c1, k4.x), tc::fma_sat(SKV_F(r, 2 * jp + 1), c1, k4.y));
+                            e2 = tc::exp2_from_unit2(y.x, y.y);
+                        } else {
+                            const uint64_t x2 = tc::ffma2(tc::pack2(SKV_F(r, 2 * jp), SKV_F(r, 2 * jp + 1)), sc2, tc::pack2(k4.x, k4.y));
+                            float xa, xb;
+                            tc::unpack2(x2, xa, xb);
+                            e2 = tc::pack2(ex2f(xa), ex2f(xb));
+                        }
+                        if (!plain) {                                       // after a row's own position: no weight
+                            float ea, eb;
+                            tc::unpack2(e2, ea, eb);
+                            e2 = tc::pack2(key > pl[c * 32 + 2 * jp] ? 0.f : ea, key > pl[c * 32 + 2 * jp + 1] ? 0.f : eb);
+                        }
+                        s2[jp & 1] = tc::ffma2(e2, tc::pack2(k4.z, k4.w), s2[jp & 1]);
                     }
                 }
                 float sum;

@@ -62,9 +62,10 @@ __device__ __forceinline__ float fma_sat(float a, float b, float c) {
     asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
-__device__ __forceinline__ uint64_t exp2_fma2(float sa, float sb, float c1, float c0) {
+// 2^x for two values given as y = (x + 126) / 254 in [0, 1]
+__device__ __forceinline__ uint64_t exp2_from_unit2(float ya, float yb) {
     constexpr float kMagic = 12582912.f - 126.f;
-    const uint64_t y = pack2(fma_sat(sa, c1, c0), fma_sat(sb, c1, c0));
+    const uint64_t y = pack2(ya, yb);
     const uint64_t t = ffma2(y, pack2(254.f, 254.f), pack2(kMagic, kMagic));
     const uint64_t fl = fadd2(t, pack2(-kMagic, -kMagic));
     const uint64_t g = ffma2(y, pack2(-254.f, -254.f), fl);
@@ -76,6 +77,9 @@ __device__ __forceinline__ uint64_t exp2_fma2(float sa, float sb, float c1, floa
     unpack2(t, ta, tb);
     return pack2(__uint_as_float(__float_as_uint(qa) + (__float_as_uint(ta) << 23)),
                  __uint_as_float(__float_as_uint(qb) + (__float_as_uint(tb) << 23)));
+}
+__device__ __forceinline__ uint64_t exp2_fma2(float sa, float sb, float c1, float c0) {
+    return exp2_from_unit2(fma_sat(sa, c1, c0), fma_sat(sb, c1, c0));
 }
 
 // Is column pair j (of 16) of a 32-column chunk exponentiated on the FMA pipe?  NP pairs are, spread evenly.

@@ -372,10 +372,10 @@ int tc_setup(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const 
 template <int D, int MB>
 int launch_colsum_tc_t(shotkv_ctx* ctx, const TcSetup& t, const ColsumTcParams& cp, cudaStream_t stream) {
     constexpr int smem = ColsumTcCfg<D, MB>::kSmemBytes;
-    CUDA_TRY(ctx, cudaFuncSetAttribute(colsum_tc_kernel<D, MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    CUDA_TRY(ctx, cudaFuncSetAttribute(colsum_tc_kernel<D, MB, kPolyEvery>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     int grid = cp.base.total_items < ctx->sm_count ? cp.base.total_items : ctx->sm_count;
     if (grid < 1) grid = 1;
-    colsum_tc_kernel<D, MB><<<grid, ColsumTcCfg<D, MB>::kThreads, smem, stream>>>(t.tmQ, t.tmK, t.qbox, t.kbox, cp);
+    colsum_tc_kernel<D, MB, kPolyEvery><<<grid, ColsumTcCfg<D, MB>::kThreads, smem, stream>>>(t.tmQ, t.tmK, t.qbox, t.kbox, cp);
     LAUNCH_CHECK(ctx);
     return SHOTKV_OK;
 }
