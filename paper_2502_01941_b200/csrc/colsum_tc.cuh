@@ -123,6 +123,7 @@ __global__ void __launch_bounds__(ColsumTcCfg<D, MB>::kThreads, 1)
         const int r0 = g * RG;                             // first window row (accumulator column) of this group
         const float scale = p.scale_log2;
         const uint64_t sc2 = tc::pack2(scale, scale);
+        const float c1 = scale * (1.f / 254.f);
         float4* cu = cst + e * (RG / 2);                   // this warp's own copy of its rows' constants
         int* pl = plim_s + e * RG;
         int acc = 0, cur_u = -1, ntile = 0;
@@ -177,26 +178,31 @@ __global__ void __launch_bounds__(ColsumTcCfg<D, MB>::kThreads, 1)
                         __syncwarp();
                         if (lane == 0) tc::mbar_arrive(pp.tempty(acc, 0));
                     }
-                    const float c1 = scale * (1.f / 254.f);
-#pragma unroll
-                    for (int jp = 0; jp < 16; ++jp) {
+                    // alpha of the pair of rows (2 jp, 2 jp + 1) at this thread's key, times 1/Z, added to the sums
+                    auto pair_term = [&](int jp, bool masked) {
                         const float4 k4 = cu[c * 16 + jp];
                         uint64_t e2;
                         if (tc::pair_on_fma<PE>(jp)) {
-                            const float2 y = make_float2(tc::fma_sat(SKV_F(r, 2 * jp), c1, k4.x), tc::fma_sat(SKV_F(r, 2 * jp + 1), c1, k4.y));
-                            e2 = tc::exp2_from_unit2(y.x, y.y);
+                            e2 = tc::exp2_from_unit2(tc::fma_sat(SKV_F(r, 2 * jp), c1, k4.x), tc::fma_sat(SKV_F(r, 2 * jp + 1), c1, k4.y));
                         } else {
                             const uint64_t x2 = tc::ffma2(tc::pack2(SKV_F(r, 2 * jp), SKV_F(r, 2 * jp + 1)), sc2, tc::pack2(k4.x, k4.y));
                             float xa, xb;
                             tc::unpack2(x2, xa, xb);
                             e2 = tc::pack2(ex2f(xa), ex2f(xb));
                         }
-                        if (!plain) {                                       // after a row's own position: no weight
+                        if (masked) {                                       // after a row's own position: no weight
                             float ea, eb;
                             tc::unpack2(e2, ea, eb);
                             e2 = tc::pack2(key > pl[c * 32 + 2 * jp] ? 0.f : ea, key > pl[c * 32 + 2 * jp + 1] ? 0.f : eb);
                         }
                         s2[jp & 1] = tc::ffma2(e2, tc::pack2(k4.z, k4.w), s2[jp & 1]);
+                    };
+                    if (plain) {
+#pragma unroll
+                        for (int jp = 0; jp < 16; ++jp) pair_term(jp, false);
+                    } else {
+#pragma unroll
+                        for (int jp = 0; jp < 16; ++jp) pair_term(jp, true);
                     }
                 }
                 float sum;
