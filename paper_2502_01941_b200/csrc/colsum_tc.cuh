@@ -113,6 +113,16 @@ __global__ void __launch_bounds__(ColsumTcCfg<D, MB>::kThreads, 1)
     const int item_begin = (int)(total * blockIdx.x / gridDim.x);
     const int item_end = (int)(total * (blockIdx.x + 1) / gridDim.x);
 
+    // Every window row is a column of the accumulator and all columns are summed by one thread, so
+    // the rows of the Q area that no copy ever writes (fewer than 128 query rows in all) must hold
+    // numbers: zero the area once, and make that visible to the tensor core's reads.
+    {
+        unsigned char* q_area = smem_raw + (pp.sQ - smem_u32(smem_raw));
+        for (int i = threadIdx.x * 16; i < Cfg::kQBytes; i += blockDim.x * 16) *reinterpret_cast<uint4*>(q_area + i) = make_uint4(0, 0, 0, 0);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncthreads();
+    }
+
     if (warp == 0) {
         if (lane == 0) tc::producer_role<D, MB, false, true>(pp, &tmQ, &tmK, q_box_rows, k_box_rows, p, item_begin, item_end);
     } else if (warp == 1 || warp == 2) {
