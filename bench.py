@@ -43,7 +43,7 @@ UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the scoring kernel per algorithmic K byte, from the ncu capture summarised in
 # profiles/score_fast_kernel_cfg3_B1_L8.md; set to None whenever the kernel changes after the capture.
-SCORE_TC_TRAFFIC_RATIO = 1.047
+SCORE_TC_TRAFFIC_RATIO = 1.044
 DECODE_TRAFFIC_RATIO = 1.012    # profiles/decode_score_kernel_cfg4_B2.md
 DECODE_ATTEND_TRAFFIC_RATIO = 1.006    # profiles/decode_attend_kernel_cfg4_B2.md
 NOMINAL_HBM_GBS = 8000.0
@@ -230,7 +230,7 @@ def run_ours(args):
                 "achieved": round(achieved, 1), "peak": peak, "peak_source": peak_src, "unit": "GB/s",
                 "frac": round(achieved / peak, 4),
                 # dram__bytes_read+write of this kernel on the B=1, L=8 copy of the workload (profiles/
-                # score_fast_kernel_cfg3_B1_L8.md: 1.047 x its K bytes), scaled by the K bytes of a full launch
+                # score_fast_kernel_cfg3_B1_L8.md: 1.044 x its K bytes), scaled by the K bytes of a full launch
                 "traffic": int(SCORE_TC_TRAFFIC_RATIO * ab["k_read"]) if SCORE_TC_TRAFFIC_RATIO and args.scoring == "fast" else None,
                 "algorithmic_bytes_per_launch": ab["k_read"], "ms_per_launch": round(score_ms, 4),
                 # what actually limits this kernel: one exponential per logit.  16 per clock per SM is what
