@@ -1,5 +1,9 @@
 // Window attention scoring on the 5th-generation tensor cores (tcgen05.mma, accumulators in
-// tensor memory) with K streamed by TMA: the STATS pass of the scoring step.
+// tensor memory) with K streamed by TMA: the exact scoring kernel (a running maximum per row),
+// and the parts every tensor-core pass of this library shares -- PTX wrappers, the shared-memory
+// and barrier map (tc::Pipe), the TMA producer and the MMA issuer (tc::producer_role,
+// tc::mma_role).  The prefill path runs score_fast.cuh first and this kernel as its repair
+// launch; with SHOTKV_SCORING_EXACT this kernel does all the work.
 //
 // Persistent CTAs, one per SM, each owning a contiguous range of work items.  An item is one
 // (unit, chunk): unit = prompt x layer x kv head, chunk = a run of whole 128-key tiles of that
