@@ -2,13 +2,15 @@
 // issuer, work items and per-(piece, window row) outputs (m, z) as score_tc.cuh, with an epilogue
 // arranged for throughput.
 //
-//   * Sixteen epilogue warps, every thread one window row and one column slice of a tile (64 of
-//     128 columns with two row blocks, 32 with one), as in the exact kernel.  When a piece is
-//     complete the warps of the later slices hand their (m, z) to the warp of slice 0 through a
-//     small ring of shared-memory slots guarded by mbarriers, so no warp waits for another at a
-//     piece end unless it is a whole ring ahead of it.  The code of the inner loop is
-//     kept small (one copy of the chunk arithmetic, one of the boundary handling): the warps of
-//     three roles share the instruction cache.
+//   * Eight epilogue warps of up to 168 registers.  With 256 window rows a warp group owns a row
+//     block and every thread one whole row of a tile (four tensor-memory loads of 32 columns),
+//     so a piece's (m, z) is written by one thread with no exchange.  With 128 rows the two
+//     groups split a tile's columns in halves; when a piece is complete the second group hands
+//     its (m, z) to the first through a small ring of shared-memory slots guarded by mbarriers,
+//     so no warp waits for another at a piece end unless it is a whole ring ahead of it.  The
+//     code of the inner loop is kept small and free of branches (one copy of the chunk
+//     arithmetic, one of the boundary handling): the warps of three roles share the
+//     instruction cache.
 //   * No running maximum.  The reference exponent m of a (row, work item) is fixed from the
 //     item's first tile: that tile's row maximum lands on 2^-32, and every later logit of the
 //     item is exponentiated against the same m.  fp32 leaves about 2^+158 above that point and
