@@ -166,7 +166,9 @@ SHOTKV_API int shotkv_compact_kv(shotkv_ctx* ctx, const shotkv_dims* dims,
  * SHOTKV_FLAG_TOKEN_IMPORTANCE the shot scores are formed directly from per-shot partial sums
  * (K is streamed once and per-token importance is never materialised; token_importance is
  * ignored and may be NULL); with it the call equals the three calls above in sequence.
- * Arguments as in those calls.  */
+ * When the units are short (fewer than 40 tokens on average, e.g. sentence-sized units or fixed
+ * chunks) the call also goes through per-token importances, kept in the workspace: the cost of
+ * that route does not grow with S.  Arguments as in those calls.  */
 SHOTKV_API int shotkv_prefill_compress(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_policy* policy,
                             const shotkv_bf16* Qwin, const shotkv_bf16* K, const shotkv_bf16* V,
                             const int32_t* offsets_host,

@@ -138,7 +138,15 @@ int check_offsets(const shotkv_dims* d, const shotkv_policy* p, const int32_t* o
 }
 
 int rpad_of(const shotkv_dims* d) { return (d->H / d->Hkv) * d->W <= 128 ? 128 : 256; }
-int pmax_of(const shotkv_dims* d) { return d->S + 2 + kMaxChunks + 1; }
+// Units shorter than this many tokens on average put a piece end in most 32-column chunks of the
+// scoring pass and make its per-piece partials a sizeable fraction of K; the fused call then goes
+// through per-token importances instead (two passes over K, cost independent of S), which
+// measures faster from about this point on.
+constexpr int kTokenRouteBelowMeanLen = 40;
+bool token_route(const shotkv_dims* d) { return d->S > 0 && (long long)d->N < (long long)kTokenRouteBelowMeanLen * d->S; }
+// Pieces per prompt the workspace is sized for: shot boundaries plus chunk ends, or chunk ends alone
+// when the shot-aware scoring pass is never run for these dims.
+int pmax_of(const shotkv_dims* d) { return (token_route(d) ? 0 : d->S) + 2 + kMaxChunks + 1; }
 
 struct PrefillWs {
     int* off;          // [B][S+1]
@@ -150,6 +158,7 @@ struct PrefillWs {
     float* row_m;      // [U][Rpad]
     float* row_invz;
     float* unit_shot;  // [U][S]
+    float* imp;        // [U][N] per-token importances of the fused call's per-token route (absent otherwise)
     int* redo;         // [1 + U * kMaxChunks] word 0: some item is marked; then one word per item the exact kernel must recompute
     size_t total;
 };
@@ -168,6 +177,7 @@ PrefillWs carve(const shotkv_dims* d, void* base) {
     w.row_m = (float*)take(U * R * 4);
     w.row_invz = (float*)take(U * R * 4);
     w.unit_shot = (float*)take(U * (size_t)(d->S > 0 ? d->S : 1) * 4);
+    w.imp = (float*)take(token_route(d) ? U * (size_t)d->N * 4 : 0);
     w.redo = (int*)take((U * kMaxChunks + 1) * 4);
     w.total = o;
     return w;
@@ -712,6 +722,21 @@ int shotkv_prefill_compress(shotkv_ctx* ctx, const shotkv_dims* dims, const shot
     }
     const char* why = "";
     if ((rc = check_dims(dims, &why))) return fail(ctx, rc, "%s", why);
+    if (token_route(dims)) {
+        // many short units: the same three steps through per-token importances held in the workspace
+        if ((rc = check_ws(ctx, dims, ws, ws_bytes))) return rc;
+        const PrefillWs w = carve(dims, ws);
+        prof_begin(ctx);
+        if ((rc = shotkv_prefill_score(ctx, dims, Qwin, K, w.imp, ws, ws_bytes, stream_)) < 0) return rc;
+        prof_mark(ctx, (cudaStream_t)stream_);
+        const int src = shotkv_select_shots(ctx, dims, policy, w.imp, offsets_host, shot_scores, keep, kept_idx, kept_count,
+                                            Mcap, ws, ws_bytes, stream_);
+        if (src < 0) return src;
+        prof_mark(ctx, (cudaStream_t)stream_);
+        if ((rc = shotkv_compact_kv(ctx, dims, K, V, kept_idx, kept_count, Mcap, Kc, Vc, stream_)) < 0) return rc;
+        prof_mark(ctx, (cudaStream_t)stream_);
+        return src;
+    }
     if ((rc = check_policy_prefill(policy, &why))) return fail(ctx, rc, "%s", why);
     int worst = 0;
     const int orc = check_offsets(dims, policy, offsets_host, &worst, &why);
