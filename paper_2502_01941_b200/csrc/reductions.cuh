@@ -112,23 +112,26 @@ __global__ void shot_score_from_mass_kernel(const float* __restrict__ unit_shot,
     }
 }
 
-// Score(s_i) from per-token importance: one CTA per (b, l, shot); fixed summation order.
-__global__ void __launch_bounds__(128) shot_score_from_tokens_kernel(const float* __restrict__ imp,
-                                                                    const int* __restrict__ off, int L, int Hkv, int N,
-                                                                    int S, float* __restrict__ shot_scores) {
-    __shared__ float red[4];
-    const int i = blockIdx.x, bl = blockIdx.y;
+// Score(s_i) from per-token importance: one warp per (b, l, shot), eight shots per CTA; every
+// lane sums a fixed subset of the shot's (kv head, token) pairs and the lanes are added by
+// shuffles, so the order is fixed.  (One CTA per shot spent most of its time being launched once
+// the units are sentence-sized and number in the thousands.)
+constexpr int kShotsPerCta = 8;
+__global__ void __launch_bounds__(32 * kShotsPerCta) shot_score_from_tokens_kernel(const float* __restrict__ imp,
+                                                                                   const int* __restrict__ off, int L,
+                                                                                   int Hkv, int N, int S,
+                                                                                   float* __restrict__ shot_scores) {
+    const int i = blockIdx.x * kShotsPerCta + (threadIdx.x >> 5), bl = blockIdx.y, lane = threadIdx.x & 31;
+    if (i >= S) return;
     const int b = bl / L;
     const int lo = off[(size_t)b * (S + 1) + i], hi = off[(size_t)b * (S + 1) + i + 1];
     float a = 0.f;
     for (int h = 0; h < Hkv; ++h) {
         const float* row = imp + ((size_t)bl * Hkv + h) * N;
-        for (int t = lo + threadIdx.x; t < hi; t += 128) a += row[t];
+        for (int t = lo + lane; t < hi; t += 32) a += row[t];
     }
     a = warp_sum(a);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = a;
-    __syncthreads();
-    if (threadIdx.x == 0) shot_scores[(size_t)bl * S + i] = (red[0] + red[1] + red[2] + red[3]) / (float)(hi - lo);
+    if (lane == 0) shot_scores[(size_t)bl * S + i] = a / (float)(hi - lo);
 }
 
 }  // namespace shotkv

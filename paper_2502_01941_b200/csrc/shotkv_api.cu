@@ -626,8 +626,8 @@ int shotkv_select_shots(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_p
     const PrefillWs w = carve(dims, ws);
     if ((rc = upload_small(ctx, w.off, offsets_host, (size_t)dims->B * (dims->S + 1) * 4, stream))) return rc;
     if (token_importance && dims->S > 0) {
-        dim3 grid(dims->S, dims->B * dims->L);
-        shot_score_from_tokens_kernel<<<grid, 128, 0, stream>>>(token_importance, w.off, dims->L, dims->Hkv, dims->N, dims->S, shot_scores);
+        dim3 grid((dims->S + kShotsPerCta - 1) / kShotsPerCta, dims->B * dims->L);
+        shot_score_from_tokens_kernel<<<grid, 32 * kShotsPerCta, 0, stream>>>(token_importance, w.off, dims->L, dims->Hkv, dims->N, dims->S, shot_scores);
         LAUNCH_CHECK(ctx);
     }
     if ((rc = run_select(ctx, dims, policy, w, shot_scores, keep, kept_idx, kept_count, Mcap, stream))) return rc;
@@ -684,8 +684,8 @@ int shotkv_select_shots_static(shotkv_ctx* ctx, const shotkv_dims* dims, const s
     // every entry the kernels read is overwritten here, so nothing of an earlier call survives
     if ((rc = upload_small(ctx, w.off, offsets_host, (size_t)entries * 4, stream))) return rc;
     if (token_importance && dims->S > 0) {
-        dim3 grid(dims->S, dims->B * dims->L);
-        shot_score_from_tokens_kernel<<<grid, 128, 0, stream>>>(token_importance, w.off, dims->L, dims->Hkv, dims->N, dims->S, shot_scores);
+        dim3 grid((dims->S + kShotsPerCta - 1) / kShotsPerCta, dims->B * dims->L);
+        shot_score_from_tokens_kernel<<<grid, 32 * kShotsPerCta, 0, stream>>>(token_importance, w.off, dims->L, dims->Hkv, dims->N, dims->S, shot_scores);
         LAUNCH_CHECK(ctx);
     }
     if ((rc = run_select(ctx, dims, policy, w, shot_scores, keep, kept_idx, kept_count, Mcap, stream))) return rc;
