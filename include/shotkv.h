@@ -48,6 +48,12 @@ typedef uint16_t shotkv_bf16;
 typedef struct {
     int32_t B, L, H, Hkv, d, N, W, S;
 } shotkv_dims;
+/* The paper selects per layer: one kept set for all KV heads of a layer (Section 5.1).  A kept set
+ * per KV head -- every head ranks the shots by the attention its own query group pays them, and
+ * the compressed caches become ragged across heads -- needs no other call: with the dense layouts
+ * above, a tensor of L layers x Hkv heads is also a tensor of L*Hkv "layers" of one head, so pass
+ *   { B, L * Hkv, H / Hkv, 1, d, N, W, S }
+ * with the same pointers.  Every per-layer output then has one entry per (layer, KV head).  */
 
 typedef struct {
     float   r_p;              /* prefill ratio: N_budget = floor(r_p * N) tokens per layer        */

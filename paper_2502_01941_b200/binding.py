@@ -140,6 +140,11 @@ def make_dims(B, L, H, Hkv, d, N, W, S) -> Dims:
     return Dims(B, L, H, Hkv, d, N, W, S)
 
 
+def per_head_dims(dims: Dims) -> Dims:
+    """The same tensors read as L*Hkv single-head layers: selection per KV head instead of per layer."""
+    return Dims(dims.B, dims.L * dims.Hkv, dims.H // dims.Hkv, 1, dims.d, dims.N, dims.W, dims.S)
+
+
 def make_policy(r_p=1.0, select_mode=0, r_d=1.0, recompress_every=1, protect_recent=0) -> Policy:
     return Policy(float(r_p), int(select_mode), float(r_d), int(recompress_every), int(protect_recent))
 
@@ -386,7 +391,7 @@ def alloc_prefill_outputs(dims: Dims, Mcap: int, device="cuda", token_importance
 
 
 __all__ = [n for n in dir() if n.startswith("shotkv_")] + [
-    "Context", "Dims", "Policy", "DecodeState", "ShotKVError", "make_dims", "make_policy", "alloc_prefill_outputs",
+    "Context", "Dims", "Policy", "DecodeState", "ShotKVError", "make_dims", "per_head_dims", "make_policy", "alloc_prefill_outputs",
     "OK", "ERR_INVALID_ARG", "ERR_UNSUPPORTED_SHAPE", "ERR_BAD_OFFSETS", "ERR_WORKSPACE_TOO_SMALL", "ERR_CUDA",
     "ERR_TIMEOUT", "WARN_BUDGET_BELOW_ALWAYS_KEPT", "FLAG_TOKEN_IMPORTANCE", "EXPORTS", "LIB_PATH", "lib",
     "SCORING_FAST", "SCORING_EXACT", "shotkv_set_scoring_mode", "shotkv_repaired_items",

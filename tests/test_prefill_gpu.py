@@ -358,3 +358,21 @@ def test_fixed_size_chunks_as_units(ctx):
     kept = gpu["kept_count"].cpu().numpy()
     always = pre + cfg.question_len
     assert ((kept - always) % c == 0).all() and kept.max() <= O.budget_tokens(cfg.r_p, N)
+
+
+def test_selection_per_kv_head_by_reading_heads_as_layers(ctx):
+    """One kept set per KV head: the same tensors with dims {B, L*Hkv, G, 1, ...}.  Checked against the
+    oracle run on each head's own slice; heads of one layer must be free to keep different shots."""
+    cfg = wl.PrefillConfig("per_head", B=1, L=2, H=8, Hkv=4, d=128, N=3000, W=16, S=10, shot_dist="uniform", shot_lo=150,
+                           shot_hi=350, question_len=120, r_p=0.3, cfg_id=51)
+    Q, K, V, off = wl.prefill_batch(cfg, "cuda")
+    dims = skv.per_head_dims(P.dims_of(cfg))
+    assert (dims.L, dims.H, dims.Hkv) == (cfg.L * cfg.Hkv, cfg.G, 1)
+    gpu = P.gpu_prefill(ctx, dims, Q, K, V, off, cfg.r_p, 0, "fused")
+    Qh = Q.view(cfg.B, cfg.L * cfg.Hkv, cfg.G, cfg.W, cfg.d)
+    Kh = K.view(cfg.B, cfg.L * cfg.Hkv, 1, cfg.N, cfg.d)
+    Vh = V.view(cfg.B, cfg.L * cfg.Hkv, 1, cfg.N, cfg.d)
+    ties = P.check_all_units(gpu, Qh, Kh, Vh, off, cfg.r_p)
+    assert ties <= 2
+    keep = gpu["keep"].cpu().numpy().reshape(cfg.L, cfg.Hkv, cfg.S)
+    assert any((keep[l] != keep[l][0]).any() for l in range(cfg.L)), "heads of a layer all chose alike: the case shows nothing"
