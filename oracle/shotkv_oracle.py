@@ -179,11 +179,13 @@ class DecodeOracle:
     step number of each entry; T = tokens generated so far.
     """
 
-    def __init__(self, Kc: np.ndarray, H: int, r_d: float, recompress_every: int, Vc: np.ndarray | None = None):
+    def __init__(self, Kc: np.ndarray, H: int, r_d: float, recompress_every: int, Vc: np.ndarray | None = None,
+                 protect_recent: int = 0):
         """With `Vc` (the kept prefill values, [Hkv, M, d] as numbers) every step also computes the
         attention output `last_out` [H, d]; `accumulate`/`step` then need `v_values`."""
         self.Kc = np.asarray(Kc, dtype=np.float64)
         self.Vc = None if Vc is None else np.asarray(Vc, dtype=np.float64)
+        self.P = int(protect_recent)            # entries of the last P steps are exempt from eviction (0: the paper's rule)
         self.Vf: list[np.ndarray] = []          # decode values as numbers (only when Vc is given)
         self.last_out = None
         self.Hkv, self.M, self.d = self.Kc.shape
@@ -234,8 +236,13 @@ class DecodeOracle:
         n = len(self.Kd)
         k = min(n, int(math.floor(self.r_d * self.T)))
         sc = self.acc if scores is None else list(scores)
-        order = sorted(range(n), key=lambda j: (-sc[j], j))
-        return sorted(order[:k])
+        # An option beyond the paper's rule (which protects nothing): entries generated in the last
+        # P steps are kept whatever their score -- they have had few steps to collect attention --
+        # and the older ones compete for the places that remain, max(0, k - protected).
+        safe = [j for j in range(n) if self.born[j] >= self.T - self.P] if self.P > 0 else []
+        rest = [j for j in range(n) if j not in set(safe)]
+        order = sorted(rest, key=lambda j: (-sc[j], j))
+        return sorted(safe + order[:max(0, k - len(safe))])
 
     def apply_keep(self, kept: list[int]) -> list[int]:
         """Compacts the decode region to the entries `kept` (ascending); returns the evicted ones."""

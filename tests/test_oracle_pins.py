@@ -505,3 +505,47 @@ def test_decode_attention_planted_mistakes_fail():
     dropped_last = O.decode_attention(q, K[:, :-1], V[:, :-1])
     for bad in (wrong_group, no_scale, dropped_last):
         assert np.max(np.abs(bad - good)) > 1e-3
+
+
+# ---------------------------------------------------------------- decode: protected recent entries
+def _decode_run(protect, steps=12, r_d=0.25, R=4, seed=4):
+    rng = np.random.default_rng(seed)
+    H, Hkv, M, d = 4, 2, 5, 8
+    dec = O.DecodeOracle(rng.standard_normal((Hkv, M, d)), H, r_d, R, protect_recent=protect)
+    hist = []
+    for s in range(steps):
+        dec.step(rng.standard_normal((H, d)), rng.standard_normal((Hkv, d)), rng.standard_normal((Hkv, d)))
+        hist.append(list(dec.born))
+    return dec, hist
+
+
+def test_protect_recent_zero_is_the_papers_rule_and_recent_entries_survive():
+    base, hist0 = _decode_run(0)
+    same, hist_same = _decode_run(0)
+    assert hist0 == hist_same
+    dec, hist = _decode_run(3)
+    # after every eviction (T multiple of 4) the entries of the last 3 steps are all present
+    for s, born in enumerate(hist):
+        T = s + 1
+        if T % 4 == 0:
+            assert set(range(T - 3, T)) <= set(born)
+            k = int(math.floor(0.25 * T))
+            assert len(born) == max(k, 3)          # protected ones may exceed the budget, nothing else is kept then
+    # the protected set is chosen by age alone: brute force over the last eviction
+    T = 12
+    assert sorted(hist[-1])[-3:] == [9, 10, 11]
+
+
+def test_protect_recent_hand_example_and_full_protection():
+    dec = O.DecodeOracle(np.zeros((1, 2, 2)), 2, r_d=0.5, recompress_every=4, protect_recent=1)
+    z = np.zeros
+    for _ in range(4):
+        dec.accumulate(z((2, 2)), z((1, 2)), z((1, 2)))
+    # T = 4, k = 2.  Scores: entry j was present for 4 - j steps with uniform weights over (2 + present) keys:
+    # older entries have collected more, so without protection entries 0 and 1 stay; with the last step
+    # protected, entry 3 stays and one place is left for entry 0.
+    assert dec.choose_keep() == [0, 3]
+    dec.P = 0
+    assert dec.choose_keep() == [0, 1]
+    dec.P = 10                                        # everything is recent: nothing is evicted
+    assert dec.choose_keep() == [0, 1, 2, 3]
