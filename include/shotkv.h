@@ -60,7 +60,8 @@ typedef struct {
     int32_t select_mode;      /* 0: stop at the first shot that overflows; 1: skip it and go on   */
     float   r_d;              /* decode ratio: k = floor(r_d * T) after T generated tokens        */
     int32_t recompress_every; /* decode: evict every this many steps (1 = every step)             */
-    int32_t protect_recent;   /* must be 0 (the paper's rule protects nothing)                    */
+    int32_t protect_recent;   /* decode: entries of the last this many steps are never evicted;   */
+                              /* 0 = the paper's rule, which protects nothing                     */
 } shotkv_policy;
 
 enum {
@@ -238,7 +239,9 @@ SHOTKV_API int shotkv_decode_init(shotkv_ctx* ctx, const shotkv_dims* dims, cons
  *      all decode keys together (M = kept_count[b][l]); acc[j] += sum over the H heads of the
  *      weight on decode entry j;
  *   3. if T % recompress_every == 0: keep the k = min(n_dec, floor(r_d*T)) entries greatest in
- *      (acc descending, index ascending), compacted in index order (Kd, Vd, acc, born).
+ *      (acc descending, index ascending), compacted in index order (Kd, Vd, acc, born).  With
+ *      protect_recent = P > 0 the entries generated in the last P steps are kept first, whatever
+ *      their score, and the others fill what is left of k (k is raised to P if it is smaller).
  *   q device [B][L][H][d] bf16;  k_new, v_new device [B][L][Hkv][d] bf16;
  *   Kc device [B][L][Hkv][Mcap][d] bf16;  kept_count device [B][L] i32.  */
 SHOTKV_API int shotkv_decode_step(shotkv_ctx* ctx, shotkv_decode_state* state,

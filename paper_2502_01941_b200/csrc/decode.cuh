@@ -375,8 +375,10 @@ __global__ void decode_accumulate_kernel(const float* __restrict__ partial, int 
 
 // Top-k of the n decode entries of one (b, l) by (acc descending, index ascending); writes the
 // kept positions in ascending order and compacts acc and born.  Shared: n floats + 3n ints + scan.
+// Entries born at or after `protect_from` rank before all others (an option beyond the paper's
+// rule; pass a value above every step number to protect nothing).
 __global__ void __launch_bounds__(kSelectThreads) decode_rank_kernel(float* __restrict__ acc, int* __restrict__ born,
-                                                                    int Dcap, int n, int k,
+                                                                    int Dcap, int n, int k, int protect_from,
                                                                     int* __restrict__ keep_pos) {
     extern __shared__ __align__(16) unsigned char sm[];
     float* a = reinterpret_cast<float*>(sm);
@@ -391,11 +393,12 @@ __global__ void __launch_bounds__(kSelectThreads) decode_rank_kernel(float* __re
         bs[j] = born[(size_t)bl * Dcap + j];
     }
     __syncthreads();
+    const float top = __int_as_float(0x7f800000);
     for (int j = tid; j < n; j += kSelectThreads) {
-        const float v = a[j];
+        const float v = bs[j] >= protect_from ? top : a[j];
         int rank = 0;
         for (int i = 0; i < n; ++i) {
-            const float w = a[i];
+            const float w = bs[i] >= protect_from ? top : a[i];
             rank += (w > v) || (w == v && i < j);
         }
         kf[j] = ds[j] = rank < k;

@@ -875,14 +875,17 @@ size_t shotkv_decode_workspace_bytes(const shotkv_dims* dims, int32_t Dcap) {
 }
 
 int32_t shotkv_decode_capacity(const shotkv_policy* policy, int32_t steps) {
-    if (!policy || steps < 0 || policy->recompress_every < 1 || !(policy->r_d >= 0.f)) return SHOTKV_ERR_INVALID_ARG;
+    if (!policy || steps < 0 || policy->recompress_every < 1 || !(policy->r_d >= 0.f) || policy->protect_recent < 0)
+        return SHOTKV_ERR_INVALID_ARG;
     // replay the host-side counters
     int n = 0, worst = 1;
     for (int T = 1; T <= steps; ++T) {
         ++n;
         if (n > worst) worst = n;
         if (T % policy->recompress_every == 0) {
-            const int k = (int)std::floor((double)policy->r_d * (double)T);
+            int k = (int)std::floor((double)policy->r_d * (double)T);
+            const int prot = policy->protect_recent < T ? policy->protect_recent : T;
+            if (k < prot) k = prot;
             if (k < n) n = k;
         }
     }
@@ -900,7 +903,7 @@ int shotkv_decode_init(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_po
     if (dims->H / dims->Hkv > 8) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "decode supports H/Hkv <= 8");
     if (!(policy->r_d >= 0.f) || !std::isfinite(policy->r_d)) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "r_d must be finite and >= 0");
     if (policy->recompress_every < 1) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "recompress_every must be >= 1");
-    if (policy->protect_recent != 0) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "protect_recent must be 0");
+    if (policy->protect_recent < 0) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "protect_recent must be >= 0");
     if (Dcap < 1 || Dcap > 4096) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "Dcap must be in [1, 4096]");
     if (Mcap < 0) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "Mcap must be >= 0");
     if (!Kd || !Vd || !acc || !born || !ws) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "device pointers must not be NULL");
@@ -977,11 +980,16 @@ int decode_step_impl(shotkv_ctx* ctx, shotkv_decode_state* st, const shotkv_bf16
     if (st->T % st->policy.recompress_every == 0) {
         const int n = st->n_dec;
         int k = (int)std::floor((double)st->policy.r_d * (double)st->T);
+        // entries of the last protect_recent steps are all still present (they were protected at every
+        // earlier eviction too) and are kept whatever their score; the others share what is left of k
+        const int prot = st->policy.protect_recent < st->T ? st->policy.protect_recent : st->T;
+        if (k < prot) k = prot;
         if (k > n) k = n;
         if (k < n) {
             const size_t rs = (size_t)n * 16 + (kSelectThreads + 1) * 4 + 16;
             CUDA_TRY(ctx, cudaFuncSetAttribute(decode_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
-            decode_rank_kernel<<<BL, kSelectThreads, rs, stream>>>(st->acc, st->born, st->Dcap, n, k, keep_pos);
+            decode_rank_kernel<<<BL, kSelectThreads, rs, stream>>>(st->acc, st->born, st->Dcap, n, k,
+                                                                   prot > 0 ? st->T - prot : 0x7fffffff, keep_pos);
             LAUNCH_CHECK(ctx);
             if (k > 0) {
                 dim3 grid(U, 2);

@@ -22,12 +22,12 @@ def ctx():
 
 
 class GpuDecoder:
-    def __init__(self, ctx, cfg: wl.DecodeConfig, Kc, kept_count, Dcap=None, Vc=None):
+    def __init__(self, ctx, cfg: wl.DecodeConfig, Kc, kept_count, Dcap=None, Vc=None, protect_recent=0):
         self.ctx, self.cfg = ctx, cfg
         self.Vc = Vc
         self.out = torch.zeros(cfg.B, cfg.L, cfg.H, cfg.d, dtype=torch.float32, device="cuda") if Vc is not None else None
         self.dims = skv.make_dims(cfg.B, cfg.L, cfg.H, cfg.Hkv, cfg.d, 1, 1, 0)
-        self.pol = skv.make_policy(r_d=cfg.r_d, recompress_every=cfg.recompress_every)
+        self.pol = skv.make_policy(r_d=cfg.r_d, recompress_every=cfg.recompress_every, protect_recent=protect_recent)
         self.Dcap = Dcap or skv.shotkv_decode_capacity(self.pol, cfg.steps)
         dev = "cuda"
         self.Kd = torch.zeros(cfg.B, cfg.L, cfg.Hkv, self.Dcap, cfg.d, dtype=torch.bfloat16, device=dev)
@@ -52,18 +52,18 @@ class GpuDecoder:
 OUT_RTOL, OUT_ATOL = 2e-3, 1e-6
 
 
-def lockstep(ctx, cfg, M, units, counts=None, steps=None, attend=False):
+def lockstep(ctx, cfg, M, units, counts=None, steps=None, attend=False, protect_recent=0):
     """Runs `steps` decode steps on the GPU for the whole batch and the oracle for `units`,
     comparing after every step.  With `attend` the fused attention-output step is the one run, and
     its output is compared too.  Returns the number of reported eviction ties."""
     Kc, kept = wl.random_prefill_cache(cfg, M, "cuda", counts)
     Vc = wl.random_prefill_values(cfg, M, "cuda") if attend else None
-    gpu = GpuDecoder(ctx, cfg, Kc, kept, Vc=Vc)
+    gpu = GpuDecoder(ctx, cfg, Kc, kept, Vc=Vc, protect_recent=protect_recent)
     orc = {}
     for (b, l) in units:
         m = int(kept[b, l])
         orc[(b, l)] = O.DecodeOracle(wl.bf16_to_f64(Kc[b, l, :, :m]), cfg.H, cfg.r_d, cfg.recompress_every,
-                                     Vc=wl.bf16_to_f64(Vc[b, l, :, :m]) if attend else None)
+                                     Vc=wl.bf16_to_f64(Vc[b, l, :, :m]) if attend else None, protect_recent=protect_recent)
     ties = 0
     for s in range(steps or cfg.steps):
         q, k, v = wl.decode_step_inputs(cfg, s, "cuda")
@@ -202,3 +202,12 @@ def test_decode_attend_same_scores_as_plain_step(ctx):
 def test_decode_attend_config4_shape_sampled_units(ctx):
     cfg = wl.DECODE_CONFIG
     assert lockstep(ctx, cfg, 3276, [(0, 0), (5, 9)], steps=40, attend=True) <= 2
+
+
+@pytest.mark.parametrize("protect", [3, 9, 100])
+def test_decode_protected_recent_entries(ctx, protect):
+    """An option beyond the paper's rule: the entries of the last P steps are never evicted (P below,
+    above and far above what the budget k = floor(r_d * T) leaves room for)."""
+    cfg = wl.DecodeConfig("dec_protect", B=2, L=1, H=8, Hkv=2, d=128, steps=40, r_d=0.25, recompress_every=8, cfg_id=27)
+    ties = lockstep(ctx, cfg, 64, [(0, 0), (1, 0)], protect_recent=protect)
+    assert ties <= 2
