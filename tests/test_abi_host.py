@@ -137,3 +137,23 @@ def test_scoring_work_partition_covers_every_key_once(cid):
     # without offsets: plain chunks
     nchunk, ck, pieces = skv.shotkv_plan_pieces(d, None, 148)
     assert pieces.shape[1] == nchunk and pieces[0, 0, 0] == 0 and pieces[0, -1, 1] == cfg.N
+
+
+def test_short_units_size_the_workspace_for_the_per_token_route():
+    """Below a mean unit length of 40 tokens the fused call goes through per-token importances, and
+    the workspace holds those (U*N floats) instead of softmax partials for S + 67 pieces."""
+    long_units = skv.make_dims(1, 2, 32, 8, 128, 32768, 64, 96)
+    short_units = skv.make_dims(1, 2, 32, 8, 128, 32768, 64, 1290)
+    edge_a = skv.make_dims(1, 2, 32, 8, 128, 32768, 64, 819)      # 32768 / 819 = 40.01: still the shot-aware route
+    edge_b = skv.make_dims(1, 2, 32, 8, 128, 32768, 64, 820)      # 39.96: per-token route
+    ws = {k: skv.shotkv_workspace_bytes(v) for k, v in dict(l=long_units, s=short_units, a=edge_a, b=edge_b).items()}
+    U, N, R = 2 * 8, 32768, 256
+    assert ws["s"] < ws["a"] and ws["b"] < ws["a"]
+    assert ws["b"] >= U * N * 4 and ws["b"] < U * N * 4 + U * 80 * R * 8 + (1 << 20)
+    assert ws["a"] >= U * (819 + 2) * R * 8
+
+
+def test_per_head_dims_reads_heads_as_layers():
+    d = skv.per_head_dims(skv.make_dims(2, 4, 32, 8, 128, 1024, 32, 5))
+    assert (d.B, d.L, d.H, d.Hkv, d.d, d.N, d.W, d.S) == (2, 32, 4, 1, 128, 1024, 32, 5)
+    assert skv.shotkv_validate(d, None, None) == 0
