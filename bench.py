@@ -170,6 +170,7 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     ctx = skv.Context(local)
     skv.shotkv_set_scoring_mode(ctx, skv.SCORING_EXACT if args.scoring == "exact" else skv.SCORING_FAST)
+    skv.shotkv_set_pipeline_groups(ctx, args.groups)
     peak, peak_src = measured_peaks()
 
     cfg = rank_config(wl.CONFIGS[args.workload], rank)
@@ -339,7 +340,7 @@ def e2e_leg(skv, ctx, cfg, dims, pol, Q, K, V, off, Mcap, world, dev, args) -> d
     return {"value": round(cfg.B * cfg.N * world / (ms * 1e-3), 1), "unit": UNIT, "ms_per_step": round(ms, 3),
             "steps": steps, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
             "api": "shotkv_prefill_compress_host",
-            "note": "page-locked host tensors: Q and K copied whole, V rows of kept tokens gathered in place, Kc/Vc written in place"}
+            "note": "page-locked host tensors: Q and K copied whole (K in up to four groups of units, each ahead of its scoring pass), V rows of kept tokens gathered in place, Kc/Vc written in place beside the next group's upload"}
 
 
 def decode_leg(skv, ctx, rank, world, dev, peak, args) -> dict:
@@ -508,6 +509,8 @@ def main():
                          "units of 10-40 tokens (the document-QA adaptation), or fixed chunks of 16 tokens")
     ap.add_argument("--scoring", default="fast", choices=["fast", "exact"],
                     help="scoring kernel: the default pair (fast kernel + exact repair) or the exact kernel alone")
+    ap.add_argument("--groups", type=int, default=0, choices=[0, 1, 2, 3, 4],
+                    help="groups of units the fused call pipelines (0: the library's choice; 1: no overlap of steps)")
     ap.add_argument("--no-tokens", action="store_true", help="skip the per-token-importance form of the step")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-decode", action="store_true")

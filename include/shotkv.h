@@ -175,7 +175,14 @@ SHOTKV_API int shotkv_compact_kv(shotkv_ctx* ctx, const shotkv_dims* dims,
  * ignored and may be NULL); with it the call equals the three calls above in sequence.
  * When the units are short (fewer than 40 tokens on average, e.g. sentence-sized units or fixed
  * chunks) the call also goes through per-token importances, kept in the workspace: the cost of
- * that route does not grow with S.  Arguments as in those calls.  */
+ * that route does not grow with S.  Arguments as in those calls.
+ *   Units (b, l) are independent (Algorithm 1 compresses layer by layer), so the single-pass form
+ *   can cut them into up to four groups -- whole prompts, or runs of layers when B = 1 -- and
+ *   reduce, select and compact one group on a stream the context owns while `stream` works on the
+ *   next (shotkv_set_pipeline_groups; by default only the host-buffer variant below does so).  To
+ *   the caller everything still happens on `stream`: the work starts after what was enqueued there
+ *   before the call, and what is enqueued there after the call starts once all of it has finished.
+ *   Every unit's results are the same whatever the grouping, up to fp32 summation order.  */
 SHOTKV_API int shotkv_prefill_compress(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_policy* policy,
                             const shotkv_bf16* Qwin, const shotkv_bf16* K, const shotkv_bf16* V,
                             const int32_t* offsets_host,
@@ -187,7 +194,9 @@ SHOTKV_API int shotkv_prefill_compress(shotkv_ctx* ctx, const shotkv_dims* dims,
 
 /* Same, for callers whose tensors live in HOST memory.  Copies Qwin and K to the device arena, runs
  * Phase 1 and delivers the results to the host buffers, all on `stream`; returns after
- * enqueueing.  Outputs with a NULL host pointer are not delivered.
+ * enqueueing.  Outputs with a NULL host pointer are not delivered.  On large inputs K goes up one
+ * group of units at a time, each just ahead of its scoring pass, so that later uploads run beside
+ * the gathers and write-backs of earlier groups.
  *   Page-locked buffers (cudaHostAlloc / cudaHostRegister) make the copies asynchronous, and
  *   more: V is only ever gathered (the Compress equation takes the kept tokens' rows), so a
  *   page-locked V_host is read in place by the compaction kernel -- only the kept rows cross the
@@ -290,12 +299,20 @@ SHOTKV_API int shotkv_set_scoring_mode(shotkv_ctx* ctx, int mode);
  * over the calls finished so far on this context.  A diagnostic: 0 on ordinary inputs.  */
 SHOTKV_API uint64_t shotkv_repaired_items(const shotkv_ctx* ctx);
 
+/* Groups the single-pass form of shotkv_prefill_compress pipelines its units in: 0 (default)
+ * chooses -- one group for device buffers, one per 256 MB of K (at most 4) for the host-buffer
+ * variant, where the groups overlap uploads with write-backs --, 1 runs every step on the
+ * caller's stream, 2..4 force that many groups where there are enough prompts (or layers).  A
+ * tuning and testing knob; the paper has no counterpart.  */
+SHOTKV_API int shotkv_set_pipeline_groups(shotkv_ctx* ctx, int groups);
+
 /* When enabled, shotkv_prefill_compress (single-pass form) and shotkv_decode_step record CUDA
  * events on their stream at their stage boundaries; the last 64 calls are retained.  */
 SHOTKV_API int shotkv_profile_enable(shotkv_ctx* ctx, int enable);
 /* Stage durations in milliseconds of the profiled call made `calls_back` calls ago (0 = latest);
- * waits for that call to finish.  Prefill: {scoring kernel, per-shot reduce, select, compact};
- * decode: {score kernel, accumulate+evict, -1, -1}.  Returns the number of stages or a negative
+ * waits for that call to finish.  Prefill: {scoring kernel, per-shot reduce, select, compact},
+ * each summed over the groups of a pipelined call (stages of different groups overlap, so the
+ * sum can exceed the call's duration); decode: {score kernel, accumulate+evict, -1, -1}.  Returns the number of stages or a negative
  * error. */
 SHOTKV_API int shotkv_profile_read(shotkv_ctx* ctx, int calls_back, float* stage_ms /* [4] */);
 /* Kernels launched through this context since it was created. */

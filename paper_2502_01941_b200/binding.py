@@ -33,7 +33,7 @@ EXPORTS = [
     "shotkv_host_arena_bytes", "shotkv_prefill_compress_host",
     "shotkv_decode_workspace_bytes", "shotkv_decode_capacity", "shotkv_decode_init", "shotkv_decode_step", "shotkv_decode_step_attend",
     "shotkv_profile_enable", "shotkv_profile_read", "shotkv_launch_count", "shotkv_select_shots_static", "shotkv_plan_pieces",
-    "shotkv_set_scoring_mode", "shotkv_repaired_items",
+    "shotkv_set_scoring_mode", "shotkv_repaired_items", "shotkv_set_pipeline_groups",
 ]
 
 
@@ -99,6 +99,7 @@ def lib() -> C.CDLL:
         "shotkv_profile_read": (C.c_int, [vp, C.c_int, C.POINTER(C.c_float)]),
         "shotkv_launch_count": (C.c_uint64, [vp]),
         "shotkv_set_scoring_mode": (C.c_int, [vp, C.c_int]),
+        "shotkv_set_pipeline_groups": (C.c_int, [vp, C.c_int]),
         "shotkv_repaired_items": (C.c_uint64, [vp]),
     }
     for name, (res, args) in sig.items():
@@ -356,6 +357,10 @@ def shotkv_set_scoring_mode(ctx: Context, mode: int) -> int:
     return ctx.check(lib().shotkv_set_scoring_mode(ctx._h, int(mode)))
 
 
+def shotkv_set_pipeline_groups(ctx: Context, groups: int) -> int:
+    return ctx.check(lib().shotkv_set_pipeline_groups(ctx._h, int(groups)))
+
+
 def shotkv_repaired_items(ctx: Context) -> int:
     return int(lib().shotkv_repaired_items(ctx._h))
 
@@ -394,5 +399,5 @@ __all__ = [n for n in dir() if n.startswith("shotkv_")] + [
     "Context", "Dims", "Policy", "DecodeState", "ShotKVError", "make_dims", "per_head_dims", "make_policy", "alloc_prefill_outputs",
     "OK", "ERR_INVALID_ARG", "ERR_UNSUPPORTED_SHAPE", "ERR_BAD_OFFSETS", "ERR_WORKSPACE_TOO_SMALL", "ERR_CUDA",
     "ERR_TIMEOUT", "WARN_BUDGET_BELOW_ALWAYS_KEPT", "FLAG_TOKEN_IMPORTANCE", "EXPORTS", "LIB_PATH", "lib",
-    "SCORING_FAST", "SCORING_EXACT", "shotkv_set_scoring_mode", "shotkv_repaired_items",
+    "SCORING_FAST", "SCORING_EXACT", "shotkv_set_scoring_mode", "shotkv_repaired_items", "shotkv_set_pipeline_groups",
 ]

@@ -9,6 +9,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <functional>
 #include <new>
 #include <vector>
 
@@ -29,6 +30,8 @@ constexpr int kMaxShots = 8192;
 constexpr int kStageSlots = 4;
 constexpr size_t kStageSlotBytes = 1u << 20;
 constexpr int kProfSlots = 64;
+constexpr int kMaxGroups = 4;         // most groups the fused prefill call pipelines its units in
+constexpr double kMinGroupKBytes = 256.0 * 1024 * 1024;   // least K a group of the automatic split holds
 
 inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
@@ -45,7 +48,17 @@ struct shotkv_ctx {
     bool prof = false;
     cudaEvent_t prof_ev[kProfSlots][5] = {};
     int prof_marks[kProfSlots] = {};
+    // the pipelined fused call records per group: scoring begin/end on the caller's stream, then
+    // begin, reduce end, selection end, compaction end on the stream those steps ran on
+    cudaEvent_t prof_gev[kProfSlots][kMaxGroups][6] = {};
+    int prof_groups[kProfSlots] = {};
     int prof_calls = 0;
+    // second stream of the fused prefill call: reduce + select + compact of one group of units run
+    // there while the caller's stream scores the next group
+    cudaStream_t aux = nullptr;
+    cudaEvent_t ev_fork[kMaxGroups] = {};
+    cudaEvent_t ev_join = nullptr;
+    int pipeline_groups = 0;           // 0 = chosen from the sizes
     unsigned long long launches = 0;   // kernels launched through this context
     // error word that kernels with bounded waits raise; pinned host memory mapped into the device
     int* err_host = nullptr;
@@ -85,6 +98,13 @@ void prof_begin(shotkv_ctx* ctx) {
     if (!ctx->prof) return;
     ctx->prof_calls += 1;
     ctx->prof_marks[(ctx->prof_calls - 1) % kProfSlots] = 0;
+    ctx->prof_groups[(ctx->prof_calls - 1) % kProfSlots] = 0;
+}
+void prof_gmark(shotkv_ctx* ctx, int group, int mark, cudaStream_t stream) {
+    if (!ctx->prof || ctx->prof_calls == 0) return;
+    const int slot = (ctx->prof_calls - 1) % kProfSlots;
+    if (group + 1 > ctx->prof_groups[slot]) ctx->prof_groups[slot] = group + 1;
+    cudaEventRecord(ctx->prof_gev[slot][group][mark], stream);
 }
 void prof_mark(shotkv_ctx* ctx, cudaStream_t stream) {
     if (!ctx->prof || ctx->prof_calls == 0) return;
@@ -159,7 +179,7 @@ struct PrefillWs {
     float* row_invz;
     float* unit_shot;  // [U][S]
     float* imp;        // [U][N] per-token importances of the fused call's per-token route (absent otherwise)
-    int* redo;         // [1 + U * kMaxChunks] word 0: some item is marked; then one word per item the exact kernel must recompute
+    int* redo;         // [kMaxGroups + U * kMaxChunks] per group of units: one word "some item is marked", then one word per item the exact kernel must recompute
     size_t total;
 };
 
@@ -178,7 +198,7 @@ PrefillWs carve(const shotkv_dims* d, void* base) {
     w.row_invz = (float*)take(U * R * 4);
     w.unit_shot = (float*)take(U * (size_t)(d->S > 0 ? d->S : 1) * 4);
     w.imp = (float*)take(token_route(d) ? U * (size_t)d->N * 4 : 0);
-    w.redo = (int*)take((U * kMaxChunks + 1) * 4);
+    w.redo = (int*)take((U * kMaxChunks + kMaxGroups) * 4);
     w.total = o;
     return w;
 }
@@ -438,13 +458,11 @@ int check_ws(shotkv_ctx* ctx, const shotkv_dims* d, void* ws, size_t ws_bytes) {
     return SHOTKV_OK;
 }
 
-// STATS pass over `pieces` followed by the per-row reduction; leaves part_m/part_z (and for the
-// token path row_m/row_invz) in the workspace.
-int run_stats(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const shotkv_bf16* K, const PrefillWs& w,
-              const int32_t* off_host, bool need_rows, int* P_out, cudaStream_t stream) {
+// Builds the piece lists of every prompt for `plan` and uploads them with the chunk index.
+int prepare_pieces(shotkv_ctx* ctx, const shotkv_dims* d, const int32_t* off_host, const ChunkPlan& plan, const PrefillWs& w,
+                   int* P_out, cudaStream_t stream) {
     std::vector<int2> pieces;
     std::vector<int> seg, chunk_first;
-    const ChunkPlan plan = plan_chunks(d, ctx->sm_count);
     const int P = build_pieces(d, off_host, plan, pieces, seg, chunk_first);
     if (P > pmax_of(d)) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "internal: piece count %d exceeds bound %d", P, pmax_of(d));
     int rc = upload_small(ctx, w.pieces, pieces.data(), pieces.size() * sizeof(int2), stream);
@@ -452,6 +470,18 @@ int run_stats(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const
     rc = upload_small(ctx, w.piece_seg, seg.data(), seg.size() * sizeof(int), stream);
     if (rc) return rc;
     rc = upload_small(ctx, w.chunk_first, chunk_first.data(), chunk_first.size() * sizeof(int), stream);
+    if (rc) return rc;
+    *P_out = P;
+    return SHOTKV_OK;
+}
+
+// STATS pass over `pieces` followed by the per-row reduction; leaves part_m/part_z (and for the
+// token path row_m/row_invz) in the workspace.
+int run_stats(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const shotkv_bf16* K, const PrefillWs& w,
+              const int32_t* off_host, bool need_rows, int* P_out, cudaStream_t stream) {
+    const ChunkPlan plan = plan_chunks(d, ctx->sm_count);
+    int P = 0;
+    int rc = prepare_pieces(ctx, d, off_host, plan, w, &P, stream);
     if (rc) return rc;
     const int U = d->B * d->L * d->Hkv;
     prof_mark(ctx, stream);
@@ -465,6 +495,68 @@ int run_stats(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const
     }
     *P_out = P;
     return SHOTKV_OK;
+}
+
+// ---- the fused call's pipeline over groups of units ---------------------------------------------
+// Units (b, l) are independent, so the fused call may cut them into groups -- whole prompts, or
+// runs of layers when there is one prompt -- and reduce, select and compact one group on a second
+// stream while the caller's stream works on the next.  With host buffers that hides the write-back
+// of one group's Kc/Vc behind the upload of the next group's K (the bus carries both directions at
+// once).  With device buffers it measured no gain (the scoring pass slows by what the overlapped
+// compaction takes: both draw on the same power budget and SMs) and a loss on small inputs, so
+// there the automatic choice is one group.
+struct GroupSplit {
+    int n;          // groups
+    int per;        // prompts (or layers, when by_layer) in every group but possibly the last
+    bool by_layer;  // one prompt, cut along its layers
+};
+GroupSplit plan_groups(const shotkv_ctx* ctx, const shotkv_dims* d, bool host_staged) {
+    GroupSplit g{1, 0, d->B == 1};
+    const int count = g.by_layer ? d->L : d->B;
+    int want = ctx->pipeline_groups;
+    if (want <= 0) {
+        // automatic: for host buffers one group per kMinGroupKBytes of K; otherwise one group
+        const double k_bytes = (double)d->B * d->L * d->Hkv * d->N * d->d * 2.0;
+        want = host_staged ? (int)(k_bytes / kMinGroupKBytes) : 1;
+    }
+    if (want > kMaxGroups) want = kMaxGroups;
+    if (want > count) want = count;
+    if (want < 1) want = 1;
+    g.per = (count + want - 1) / want;
+    g.n = (count + g.per - 1) / g.per;
+    return g;
+}
+// One group's share of the call: its dims, and the offsets of its first prompt, first (b, l) pair and first unit.
+struct GroupView {
+    shotkv_dims d;
+    size_t b0, bl0, u0;
+};
+GroupView group_view(const shotkv_dims* d, const GroupSplit& gs, int g) {
+    GroupView v{};
+    v.d = *d;
+    const int count = gs.by_layer ? d->L : d->B;
+    const int first = g * gs.per;
+    const int n = first + gs.per <= count ? gs.per : count - first;
+    if (gs.by_layer) { v.d.L = n; v.b0 = 0; v.bl0 = (size_t)first; }
+    else { v.d.B = n; v.b0 = (size_t)first; v.bl0 = (size_t)first * d->L; }
+    v.u0 = v.bl0 * d->Hkv;
+    return v;
+}
+// The group's slices of the workspace arrays (P = pieces per prompt as uploaded).
+PrefillWs group_ws(const PrefillWs& w, const shotkv_dims* d, const GroupView& v, int g, int P) {
+    PrefillWs x = w;
+    const size_t R = rpad_of(d);
+    x.off = w.off + v.b0 * (d->S + 1);
+    x.pieces = w.pieces + v.b0 * P;
+    x.piece_seg = w.piece_seg + v.b0 * P;
+    x.chunk_first = w.chunk_first + v.b0 * (kMaxChunks + 1);
+    x.part_m = w.part_m + v.u0 * P * R;
+    x.part_z = w.part_z + v.u0 * P * R;
+    x.row_m = w.row_m + v.u0 * R;
+    x.row_invz = w.row_invz + v.u0 * R;
+    x.unit_shot = w.unit_shot + v.u0 * (size_t)(d->S > 0 ? d->S : 1);
+    x.redo = w.redo + g + v.u0 * kMaxChunks;
+    return x;
 }
 
 int run_select(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_policy* p, const PrefillWs& w, float* shot_scores,
@@ -530,6 +622,13 @@ int shotkv_create(shotkv_ctx** out, int device) {
         shotkv_destroy(ctx);
         return SHOTKV_ERR_CUDA;
     }
+    bool ok = cudaStreamCreateWithFlags(&ctx->aux, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; ok && i < kMaxGroups; ++i) ok = cudaEventCreateWithFlags(&ctx->ev_fork[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+        shotkv_destroy(ctx);
+        return SHOTKV_ERR_CUDA;
+    }
     ctx->err_host[0] = 0;      // word 0: a bounded wait gave up
     ctx->err_host[1] = 0;      // word 1: work items the exact scoring kernel recomputed after the fast one
     ctx->sm_count = prop.multiProcessorCount;
@@ -545,11 +644,22 @@ void shotkv_destroy(shotkv_ctx* ctx) {
             cudaEventSynchronize(ctx->stage_done[i]);
             cudaEventDestroy(ctx->stage_done[i]);
         }
+    if (ctx->aux) {
+        cudaStreamSynchronize(ctx->aux);
+        cudaStreamDestroy(ctx->aux);
+    }
+    if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+    for (int i = 0; i < kMaxGroups; ++i)
+        if (ctx->ev_fork[i]) cudaEventDestroy(ctx->ev_fork[i]);
     if (ctx->stage) cudaFreeHost(ctx->stage);
     if (ctx->err_host) cudaFreeHost(ctx->err_host);
-    for (int i = 0; i < kProfSlots; ++i)
+    for (int i = 0; i < kProfSlots; ++i) {
         for (int j = 0; j < 5; ++j)
             if (ctx->prof_ev[i][j]) cudaEventDestroy(ctx->prof_ev[i][j]);
+        for (int g = 0; g < kMaxGroups; ++g)
+            for (int j = 0; j < 6; ++j)
+                if (ctx->prof_gev[i][g][j]) cudaEventDestroy(ctx->prof_gev[i][g][j]);
+    }
     delete ctx;
 }
 
@@ -705,36 +815,42 @@ int shotkv_compact_kv(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_bf1
     return run_compact(ctx, dims, K, V, kept_idx, kept_count, Mcap, Kc, Vc, (cudaStream_t)stream_);
 }
 
-int shotkv_prefill_compress(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_policy* policy, const shotkv_bf16* Qwin,
-                            const shotkv_bf16* K, const shotkv_bf16* V, const int32_t* offsets_host, float* shot_scores,
-                            uint8_t* keep, int32_t* kept_idx, int32_t* kept_count, int32_t Mcap, shotkv_bf16* Kc,
-                            shotkv_bf16* Vc, float* token_importance, uint32_t flags, void* ws, size_t ws_bytes,
-                            void* stream_) {
+namespace {
+// Called on the caller's stream before a group's scoring pass is enqueued (the host-buffer variant
+// copies that group's K there).
+using BeforeGroup = std::function<int(const GroupView&, cudaStream_t)>;
+
+int prefill_compress_impl(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_policy* policy, const shotkv_bf16* Qwin,
+                          const shotkv_bf16* K, const shotkv_bf16* V, const int32_t* offsets_host, float* shot_scores,
+                          uint8_t* keep, int32_t* kept_idx, int32_t* kept_count, int32_t Mcap, shotkv_bf16* Kc,
+                          shotkv_bf16* Vc, float* token_importance, uint32_t flags, void* ws, size_t ws_bytes,
+                          void* stream_, const BeforeGroup* before_group) {
     int rc = set_device(ctx);
     if (rc) return rc;
-    if (flags & SHOTKV_FLAG_TOKEN_IMPORTANCE) {
-        if ((rc = shotkv_prefill_score(ctx, dims, Qwin, K, token_importance, ws, ws_bytes, stream_)) < 0) return rc;
-        const int src = shotkv_select_shots(ctx, dims, policy, token_importance, offsets_host, shot_scores, keep, kept_idx,
-                                            kept_count, Mcap, ws, ws_bytes, stream_);
-        if (src < 0) return src;
-        if ((rc = shotkv_compact_kv(ctx, dims, K, V, kept_idx, kept_count, Mcap, Kc, Vc, stream_)) < 0) return rc;
-        return src;
-    }
     const char* why = "";
     if ((rc = check_dims(dims, &why))) return fail(ctx, rc, "%s", why);
-    if (token_route(dims)) {
-        // many short units: the same three steps through per-token importances held in the workspace
-        if ((rc = check_ws(ctx, dims, ws, ws_bytes))) return rc;
-        const PrefillWs w = carve(dims, ws);
-        prof_begin(ctx);
-        if ((rc = shotkv_prefill_score(ctx, dims, Qwin, K, w.imp, ws, ws_bytes, stream_)) < 0) return rc;
-        prof_mark(ctx, (cudaStream_t)stream_);
-        const int src = shotkv_select_shots(ctx, dims, policy, w.imp, offsets_host, shot_scores, keep, kept_idx, kept_count,
+    const bool tokens = (flags & SHOTKV_FLAG_TOKEN_IMPORTANCE) != 0;
+    if (tokens || token_route(dims)) {
+        // per-token importances first (asked for, or many short units): the three public steps in
+        // turn; without the flag the importances live in the workspace
+        float* imp = token_importance;
+        if (!tokens) {
+            if ((rc = check_ws(ctx, dims, ws, ws_bytes))) return rc;
+            imp = carve(dims, ws).imp;
+            prof_begin(ctx);
+        }
+        if (before_group) {
+            const GroupSplit whole{1, dims->B == 1 ? dims->L : dims->B, dims->B == 1};
+            if ((rc = (*before_group)(group_view(dims, whole, 0), (cudaStream_t)stream_))) return rc;
+        }
+        if ((rc = shotkv_prefill_score(ctx, dims, Qwin, K, imp, ws, ws_bytes, stream_)) < 0) return rc;
+        if (!tokens) prof_mark(ctx, (cudaStream_t)stream_);
+        const int src = shotkv_select_shots(ctx, dims, policy, imp, offsets_host, shot_scores, keep, kept_idx, kept_count,
                                             Mcap, ws, ws_bytes, stream_);
         if (src < 0) return src;
-        prof_mark(ctx, (cudaStream_t)stream_);
+        if (!tokens) prof_mark(ctx, (cudaStream_t)stream_);
         if ((rc = shotkv_compact_kv(ctx, dims, K, V, kept_idx, kept_count, Mcap, Kc, Vc, stream_)) < 0) return rc;
-        prof_mark(ctx, (cudaStream_t)stream_);
+        if (!tokens) prof_mark(ctx, (cudaStream_t)stream_);
         return src;
     }
     if ((rc = check_policy_prefill(policy, &why))) return fail(ctx, rc, "%s", why);
@@ -748,33 +864,77 @@ int shotkv_prefill_compress(shotkv_ctx* ctx, const shotkv_dims* dims, const shot
     if ((rc = check_ws(ctx, dims, ws, ws_bytes))) return rc;
     cudaStream_t stream = (cudaStream_t)stream_;
     const PrefillWs w = carve(dims, ws);
-    if ((rc = upload_small(ctx, w.off, offsets_host, (size_t)dims->B * (dims->S + 1) * 4, stream))) return rc;
+    const int S = dims->S, R = (dims->H / dims->Hkv) * dims->W, Rpad = rpad_of(dims);
+    const size_t S1 = S > 0 ? S : 1, row = dims->d;
+
+    // tables of all prompts once, cut for the work partition of one (full) group
+    const GroupSplit gs = plan_groups(ctx, dims, before_group != nullptr);
+    const GroupView first = group_view(dims, gs, 0);
+    const ChunkPlan plan = plan_chunks(&first.d, ctx->sm_count);
+    if ((rc = upload_small(ctx, w.off, offsets_host, (size_t)dims->B * (S + 1) * 4, stream))) return rc;
     int P = 0;
-    prof_begin(ctx);
-    if ((rc = run_stats(ctx, dims, Qwin, K, w, offsets_host, false, &P, stream))) return rc;
-    const int U = dims->B * dims->L * dims->Hkv;
-    const int R = (dims->H / dims->Hkv) * dims->W, Rpad = rpad_of(dims);
-    if (dims->S > 0) {
-        const size_t msm = (size_t)P * (Rpad / 32 + 1) * 4;
-        if (msm > 200 * 1024) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "too many shots for the single-pass path (S = %d)", dims->S);
-        if (Rpad == 128) {
-            if (msm > 48 * 1024) CUDA_TRY(ctx, cudaFuncSetAttribute(shot_mass_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)msm));
-            shot_mass_kernel<128><<<U, 128, msm, stream>>>(w.part_m, w.part_z, w.piece_seg, P, R, Rpad, dims->L, dims->Hkv, dims->S, w.unit_shot);
-        } else {
-            if (msm > 48 * 1024) CUDA_TRY(ctx, cudaFuncSetAttribute(shot_mass_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)msm));
-            shot_mass_kernel<256><<<U, 256, msm, stream>>>(w.part_m, w.part_z, w.piece_seg, P, R, Rpad, dims->L, dims->Hkv, dims->S, w.unit_shot);
+    if ((rc = prepare_pieces(ctx, dims, offsets_host, plan, w, &P, stream))) return rc;
+    const size_t msm = (size_t)P * (Rpad / 32 + 1) * 4;
+    if (S > 0) {
+        if (msm > 200 * 1024) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "too many shots for the single-pass path (S = %d)", S);
+        if (msm > 48 * 1024) {
+            if (Rpad == 128) CUDA_TRY(ctx, cudaFuncSetAttribute(shot_mass_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)msm));
+            else CUDA_TRY(ctx, cudaFuncSetAttribute(shot_mass_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)msm));
         }
-        LAUNCH_CHECK(ctx);
-        shot_score_from_mass_kernel<<<dims->B * dims->L, 128, 0, stream>>>(w.unit_shot, w.off, dims->L, dims->Hkv, dims->S, shot_scores);
-        LAUNCH_CHECK(ctx);
     }
-    prof_mark(ctx, stream);
-    if ((rc = run_select(ctx, dims, policy, w, shot_scores, keep, kept_idx, kept_count, Mcap, stream))) return rc;
-    prof_mark(ctx, stream);
-    if ((rc = run_compact(ctx, dims, K, V, kept_idx, kept_count, Mcap, Kc, Vc, stream))) return rc;
-    prof_mark(ctx, stream);
+    prof_begin(ctx);
+    const bool forked = gs.n > 1;
+    cudaStream_t tail = forked ? ctx->aux : stream;
+    for (int g = 0; g < gs.n; ++g) {
+        const GroupView v = group_view(dims, gs, g);
+        const PrefillWs wg = group_ws(w, dims, v, g, P);
+        const shotkv_dims* dg = &v.d;
+        const int Ug = dg->B * dg->L * dg->Hkv;
+        const shotkv_bf16* Kg = K + v.u0 * dims->N * row;
+        const shotkv_bf16* Vg = V + v.u0 * dims->N * row;
+        float* scores_g = shot_scores + v.bl0 * S1;
+        int32_t* idx_g = kept_idx + v.bl0 * (size_t)Mcap;
+        int32_t* count_g = kept_count + v.bl0;
+        if (before_group && (rc = (*before_group)(v, stream))) return rc;
+        prof_gmark(ctx, g, 0, stream);
+        if ((rc = launch_score_tc(ctx, dg, Qwin + v.bl0 * dims->H * dims->W * row, Kg, wg, P, plan, stream))) return rc;
+        prof_gmark(ctx, g, 1, stream);
+        if (forked) {
+            CUDA_TRY(ctx, cudaEventRecord(ctx->ev_fork[g], stream));
+            CUDA_TRY(ctx, cudaStreamWaitEvent(tail, ctx->ev_fork[g], 0));
+        }
+        prof_gmark(ctx, g, 2, tail);
+        if (S > 0) {
+            if (Rpad == 128)
+                shot_mass_kernel<128><<<Ug, 128, msm, tail>>>(wg.part_m, wg.part_z, wg.piece_seg, P, R, Rpad, dg->L, dg->Hkv, S, wg.unit_shot);
+            else
+                shot_mass_kernel<256><<<Ug, 256, msm, tail>>>(wg.part_m, wg.part_z, wg.piece_seg, P, R, Rpad, dg->L, dg->Hkv, S, wg.unit_shot);
+            LAUNCH_CHECK(ctx);
+            shot_score_from_mass_kernel<<<dg->B * dg->L, 128, 0, tail>>>(wg.unit_shot, wg.off, dg->L, dg->Hkv, S, scores_g);
+            LAUNCH_CHECK(ctx);
+        }
+        prof_gmark(ctx, g, 3, tail);
+        if ((rc = run_select(ctx, dg, policy, wg, scores_g, keep + v.bl0 * S1, idx_g, count_g, Mcap, tail))) return rc;
+        prof_gmark(ctx, g, 4, tail);
+        if ((rc = run_compact(ctx, dg, Kg, Vg, idx_g, count_g, Mcap, Kc + v.u0 * (size_t)Mcap * row, Vc + v.u0 * (size_t)Mcap * row, tail))) return rc;
+        prof_gmark(ctx, g, 5, tail);
+    }
+    if (forked) {
+        CUDA_TRY(ctx, cudaEventRecord(ctx->ev_join, tail));
+        CUDA_TRY(ctx, cudaStreamWaitEvent(stream, ctx->ev_join, 0));
+    }
     if (orc > 0) fail(ctx, orc, "always-kept tokens (%d) exceed the budget (%d) for some prompt", worst, budget_of(dims, policy));
     return orc;
+}
+}  // namespace
+
+int shotkv_prefill_compress(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_policy* policy, const shotkv_bf16* Qwin,
+                            const shotkv_bf16* K, const shotkv_bf16* V, const int32_t* offsets_host, float* shot_scores,
+                            uint8_t* keep, int32_t* kept_idx, int32_t* kept_count, int32_t Mcap, shotkv_bf16* Kc,
+                            shotkv_bf16* Vc, float* token_importance, uint32_t flags, void* ws, size_t ws_bytes,
+                            void* stream_) {
+    return prefill_compress_impl(ctx, dims, policy, Qwin, K, V, offsets_host, shot_scores, keep, kept_idx, kept_count, Mcap, Kc,
+                                 Vc, token_importance, flags, ws, ws_bytes, stream_, nullptr);
 }
 
 // ---- host-buffer variant -------------------------------------------------------------------
@@ -848,14 +1008,21 @@ int shotkv_prefill_compress_host(shotkv_ctx* ctx, const shotkv_dims* dims, const
     shotkv_bf16* Vc_out = (shotkv_bf16*)device_alias(Vc_host);
     if (((uintptr_t)V_in | (uintptr_t)Kc_out | (uintptr_t)Vc_out) & 15) V_in = nullptr, Kc_out = Vc_out = nullptr;
     CUDA_TRY(ctx, cudaMemcpyAsync(a.Q, Qwin_host, BL * dims->H * dims->W * dims->d * 2, cudaMemcpyHostToDevice, stream));
-    CUDA_TRY(ctx, cudaMemcpyAsync(a.K, K_host, U * dims->N * dims->d * 2, cudaMemcpyHostToDevice, stream));
+    // K goes up one group of units at a time, just ahead of that group's scoring pass, so that the
+    // copies of later groups run beside the gathers and write-backs of earlier ones
+    const size_t unit_elems = (size_t)dims->N * dims->d;
+    const BeforeGroup copy_k = [&](const GroupView& v, cudaStream_t s) -> int {
+        const size_t units = (size_t)v.d.B * v.d.L * v.d.Hkv;
+        CUDA_TRY(ctx, cudaMemcpyAsync(a.K + v.u0 * unit_elems, K_host + v.u0 * unit_elems, units * unit_elems * 2, cudaMemcpyHostToDevice, s));
+        return SHOTKV_OK;
+    };
     if (!V_in) {
         CUDA_TRY(ctx, cudaMemcpyAsync(a.V, V_host, U * dims->N * dims->d * 2, cudaMemcpyHostToDevice, stream));
         V_in = a.V;
     }
-    const int prc = shotkv_prefill_compress(ctx, dims, policy, a.Q, a.K, V_in, offsets_host, a.scores, a.keep, a.idx, a.count,
-                                            Mcap, Kc_out ? Kc_out : a.Kc, Vc_out ? Vc_out : a.Vc, nullptr, 0, a.ws,
-                                            a.ws_bytes, stream_);
+    const int prc = prefill_compress_impl(ctx, dims, policy, a.Q, a.K, V_in, offsets_host, a.scores, a.keep, a.idx, a.count,
+                                          Mcap, Kc_out ? Kc_out : a.Kc, Vc_out ? Vc_out : a.Vc, nullptr, 0, a.ws,
+                                          a.ws_bytes, stream_, &copy_k);
     if (prc < 0) return prc;
     const size_t S1 = dims->S > 0 ? dims->S : 1;
     if (shot_scores_host) CUDA_TRY(ctx, cudaMemcpyAsync(shot_scores_host, a.scores, BL * S1 * 4, cudaMemcpyDeviceToHost, stream));
@@ -1057,12 +1224,23 @@ int shotkv_set_scoring_mode(shotkv_ctx* ctx, int mode) {
     return SHOTKV_OK;
 }
 
+int shotkv_set_pipeline_groups(shotkv_ctx* ctx, int groups) {
+    if (!ctx) return SHOTKV_ERR_INVALID_ARG;
+    if (groups < 0 || groups > kMaxGroups)
+        return fail(ctx, SHOTKV_ERR_INVALID_ARG, "pipeline groups must be 0 (automatic) or 1..%d", kMaxGroups);
+    ctx->pipeline_groups = groups;
+    return SHOTKV_OK;
+}
+
 int shotkv_profile_enable(shotkv_ctx* ctx, int enable) {
     int rc = set_device(ctx);
     if (rc) return rc;
     if (enable && !ctx->prof_ev[0][0]) {
-        for (int i = 0; i < kProfSlots; ++i)
+        for (int i = 0; i < kProfSlots; ++i) {
             for (int j = 0; j < 5; ++j) CUDA_TRY(ctx, cudaEventCreate(&ctx->prof_ev[i][j]));
+            for (int g = 0; g < kMaxGroups; ++g)
+                for (int j = 0; j < 6; ++j) CUDA_TRY(ctx, cudaEventCreate(&ctx->prof_gev[i][g][j]));
+        }
     }
     ctx->prof = enable != 0;
     ctx->prof_calls = 0;
@@ -1077,6 +1255,22 @@ int shotkv_profile_read(shotkv_ctx* ctx, int calls_back, float* stage_ms) {
     const int slot = (ctx->prof_calls - 1 - calls_back) % kProfSlots;
     const int m = ctx->prof_marks[slot];
     for (int i = 0; i < 4; ++i) stage_ms[i] = -1.f;
+    if (const int ng = ctx->prof_groups[slot]) {
+        // pipelined fused call: each stage's time summed over the groups (the stages of different
+        // groups overlap, so the sum may exceed the call's wall time)
+        CUDA_TRY(ctx, cudaEventSynchronize(ctx->prof_gev[slot][ng - 1][5]));
+        static const int from[4] = {0, 2, 3, 4};
+        for (int i = 0; i < 4; ++i) {
+            float sum = 0.f;
+            for (int g = 0; g < ng; ++g) {
+                float ms = 0.f;
+                CUDA_TRY(ctx, cudaEventElapsedTime(&ms, ctx->prof_gev[slot][g][from[i]], ctx->prof_gev[slot][g][from[i] + 1]));
+                sum += ms;
+            }
+            stage_ms[i] = sum;
+        }
+        return 4;
+    }
     if (m < 2) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "that call recorded no stages");
     CUDA_TRY(ctx, cudaEventSynchronize(ctx->prof_ev[slot][m - 1]));
     for (int i = 0; i + 1 < m; ++i) CUDA_TRY(ctx, cudaEventElapsedTime(&stage_ms[i], ctx->prof_ev[slot][i], ctx->prof_ev[slot][i + 1]));

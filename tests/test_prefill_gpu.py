@@ -376,3 +376,79 @@ def test_selection_per_kv_head_by_reading_heads_as_layers(ctx):
     assert ties <= 2
     keep = gpu["keep"].cpu().numpy().reshape(cfg.L, cfg.Hkv, cfg.S)
     assert any((keep[l] != keep[l][0]).any() for l in range(cfg.L)), "heads of a layer all chose alike: the case shows nothing"
+
+
+GROUPED = [
+    # three prompts: groups of whole prompts (2 groups: 2 + 1 prompts; 3 or 4 asked: one prompt each)
+    wl.CONFIGS[3].replace(name="three_prompts", B=3, L=2, N=1700, S=6, shot_lo=150, shot_hi=300, question_len=120),
+    # one prompt, five layers: runs of layers (2 groups: 3 + 2 layers; 3 or 4 asked: 2 + 2 + 1)
+    wl.CONFIGS[2].replace(name="five_layers", L=5, N=1500, S=5, shot_lo=100, shot_hi=300, question_len=100),
+]
+
+
+@pytest.mark.parametrize("groups", [2, 3, 4])
+@pytest.mark.parametrize("cfg", GROUPED, ids=[c.name for c in GROUPED])
+def test_pipelined_groups_of_units(ctx, cfg, groups):
+    """The fused call with its units cut into groups, the later steps of one group running beside
+    the scoring of the next: same results as the definition, for even and uneven groups."""
+    skv.shotkv_set_pipeline_groups(ctx, groups)
+    try:
+        ties, _ = run_cfg(ctx, cfg, "fused")
+    finally:
+        skv.shotkv_set_pipeline_groups(ctx, 0)
+    assert ties <= 2
+
+
+def test_pipelined_call_is_ordered_on_the_callers_stream(ctx):
+    """Work enqueued on the caller's stream right after a pipelined call sees all of its outputs, and
+    a second call may reuse workspace and outputs at once."""
+    cfg = GROUPED[0]
+    Q, K, V, off = wl.prefill_batch(cfg, "cuda")
+    dims = P.dims_of(cfg)
+    pol = skv.make_policy(r_p=cfg.r_p)
+    Mcap = skv.shotkv_kept_capacity(dims, pol, off)
+    out = skv.alloc_prefill_outputs(dims, Mcap)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    skv.shotkv_set_pipeline_groups(ctx, 3)
+    try:
+        snaps = []
+        with torch.cuda.stream(side):
+            for _ in range(3):
+                for k in ("shot_scores", "keep", "kept_idx", "kept_count", "Kc", "Vc"):
+                    out[k].zero_()
+                skv.shotkv_prefill_compress(ctx, dims, pol, Q, K, V, off, out["shot_scores"], out["keep"], out["kept_idx"],
+                                            out["kept_count"], Mcap, out["Kc"], out["Vc"], None, 0, out["ws"])
+                snaps.append({k: out[k].clone() for k in ("shot_scores", "keep", "kept_idx", "kept_count", "Kc", "Vc")})
+        side.synchronize()
+    finally:
+        skv.shotkv_set_pipeline_groups(ctx, 0)
+    for snap in snaps:
+        snap["token_importance"] = None
+        P.check_all_units(snap, Q, K, V, off, cfg.r_p)
+    for k in snaps[0]:
+        if k != "token_importance":
+            assert torch.equal(snaps[0][k], snaps[2][k]), k
+
+
+def test_host_buffer_entry_point_pipelined(ctx):
+    """Host buffers with the units in groups: K goes up group by group ahead of each scoring pass."""
+    cfg = SHRUNK[1]
+    Q, K, V, off = wl.prefill_batch(cfg, "cpu")
+    dims = P.dims_of(cfg)
+    pol = skv.make_policy(r_p=cfg.r_p)
+    Mcap = skv.shotkv_kept_capacity(dims, pol, off)
+    hout = skv.alloc_prefill_outputs(dims, Mcap, device="cpu")
+    for k in ("shot_scores", "keep", "kept_idx", "kept_count", "Kc", "Vc"):
+        hout[k] = hout[k].pin_memory()
+    arena = torch.zeros(skv.shotkv_host_arena_bytes(dims, Mcap), dtype=torch.uint8, device="cuda")
+    skv.shotkv_set_pipeline_groups(ctx, 2)
+    try:
+        skv.shotkv_prefill_compress_host(ctx, dims, pol, Q.pin_memory(), K.pin_memory(), V.pin_memory(), off,
+                                         hout["shot_scores"], hout["keep"], hout["kept_idx"], hout["kept_count"], Mcap,
+                                         hout["Kc"], hout["Vc"], arena)
+        torch.cuda.synchronize()
+    finally:
+        skv.shotkv_set_pipeline_groups(ctx, 0)
+    hout["token_importance"] = None
+    P.check_all_units(hout, Q, K, V, off, cfg.r_p)
