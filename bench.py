@@ -41,12 +41,15 @@ from paper_2502_01941_b200 import workloads as wl
 METRIC = "prompt tokens compressed/sec"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
-# DRAM traffic of the scoring kernel per algorithmic K byte, from the ncu capture summarised in
-# profiles/score_fast_kernel_cfg3_B1_L8.md; set to None whenever the kernel changes after the capture.
-SCORE_TC_TRAFFIC_RATIO = 1.044
-DECODE_TRAFFIC_RATIO = 1.012    # profiles/decode_score_kernel_cfg4_B2.md
-DECODE_ATTEND_TRAFFIC_RATIO = 1.006    # profiles/decode_attend_kernel_cfg4_B2.md
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, one ncu capture each) per algorithmic
+# byte of the scoring kernel and of the two decode score kernels, taken on reduced copies of the
+# workloads (config 3 with B=1, L=8; config 4 with B=2) and scaled by the bytes of a full launch.
+# A ratio is set to None whenever its kernel has changed since its capture.
+SCORE_TC_TRAFFIC_RATIO = None
+DECODE_TRAFFIC_RATIO = 1.012
+DECODE_ATTEND_TRAFFIC_RATIO = None
 NOMINAL_HBM_GBS = 8000.0
+SUSTAIN_SECONDS = 2.5           # length of the sustained repeat of the step
 
 
 # ------------------------------------------------------------------ small utilities
@@ -223,22 +226,37 @@ def run_ours(args):
     value = tokens / (ms_step * 1e-3)
     achieved = ab["k_read"] / (score_ms * 1e-3) / 1e9
     logits = cfg.B * cfg.L * cfg.H * cfg.W * cfg.N                       # one ex2 per window logit
-    sm_mhz = clocks.get("sm_mhz") or 1965.0
-    ex2_rate = logits / (score_ms * 1e-3) / 148 / (sm_mhz * 1e6)
+    sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+    tiles_per_sm = cfg.B * cfg.L * cfg.Hkv * ((cfg.N + 127) // 128) / sm_count
+    # ---------------- the same step repeated for seconds: what the path sustains once the clock has
+    # settled under the power cap (the --steps figure above may be a burst of a few tens of ms)
+    sustained = None
+    if not args.no_sustained:
+        sustained = sustained_leg(skv, ctx, step, ms_step, cfg, ab, peak, tiles_per_sm, world, dev, local)
+    # host copies of prompt 0's results, for the parity record taken beside the CPU baseline
+    gpu_prompt0 = {k: out[k][0].cpu() for k in ("shot_scores", "keep", "kept_idx", "kept_count")}
+    gpu_prompt0["Kc"] = out["Kc"][0, :PARITY_ROW_UNITS].cpu()
+    gpu_prompt0["Vc"] = out["Vc"][0, :PARITY_ROW_UNITS].cpu()
+    # the per-clock rate is taken at the clock of the sustained region when there is one (tens of
+    # samples), else at the clock sampled during the --steps region
+    sm_mhz = (sustained or {}).get("clocks", {}).get("sm_mhz") or clocks.get("sm_mhz") or 1965.0
+    rate_ms = sustained["stage_ms"]["score"] if sustained else score_ms
+    ex2_rate = logits / (rate_ms * 1e-3) / sm_count / (sm_mhz * 1e6)
     kernel_name = ("score_fast_kernel" if args.scoring == "fast" else "score_tc_kernel") + \
         " (window QK^T on tcgen05 + softmax partials), one launch per step"
     roofline = {"bound": "hbm", "kernel": kernel_name,
                 "achieved": round(achieved, 1), "peak": peak, "peak_source": peak_src, "unit": "GB/s",
                 "frac": round(achieved / peak, 4),
-                # dram__bytes_read+write of this kernel on the B=1, L=8 copy of the workload (profiles/
-                # score_fast_kernel_cfg3_B1_L8.md: 1.044 x its K bytes), scaled by the K bytes of a full launch
+                # measured DRAM bytes per launch: the captured ratio times the K bytes of a full launch
                 "traffic": int(SCORE_TC_TRAFFIC_RATIO * ab["k_read"]) if SCORE_TC_TRAFFIC_RATIO and args.scoring == "fast" else None,
                 "algorithmic_bytes_per_launch": ab["k_read"], "ms_per_launch": round(score_ms, 4),
                 # what actually limits this kernel: one exponential per logit.  16 per clock per SM is what
                 # the special-function unit alone delivers (measured); the kernel takes 5 of every 16
                 # column pairs on the FMA pipe instead, so the fraction may pass 1
                 "also": {"bound": "alu", "unit": "exp/clk/SM", "achieved": round(ex2_rate, 2), "peak": 16.0,
-                         "frac": round(ex2_rate / 16.0, 4), "at_sm_mhz": sm_mhz}}
+                         "frac": round(ex2_rate / 16.0, 4), "at_sm_mhz": sm_mhz,
+                         "cycles_per_tile": round(rate_ms * 1e-3 * sm_mhz * 1e6 / tiles_per_sm, 1),
+                         "region": "sustained" if sustained else "steps"}}
     path = {"bytes_per_step": ab["total"], "k_read_bytes": ab["k_read"], "kv_gathered_bytes": ab["kv_gathered"],
             "achieved_gbs": round(ab["total"] / (ms_step * 1e-3) / 1e9, 1),
             "frac_of_measured_hbm": round(ab["total"] / (ms_step * 1e-3) / 1e9 / peak, 4),
@@ -257,6 +275,8 @@ def run_ours(args):
                    "parallelism": f"{world} independent replica(s), one batch of prompts each"},
         "roofline": roofline, "path": path, "clocks": clocks, "gpu_launches": int(launches),
     }
+    if sustained:
+        result["sustained"] = sustained
 
     # ---------------- the per-token form of the step (shotkv_prefill_score: a second pass over K
     # that normalises and column-sums, then selection from token importances, then compaction)
@@ -290,7 +310,7 @@ def run_ours(args):
         result["decode"] = decode_leg(skv, ctx, rank, world, dev, peak, args)
     # ---------------- CPU baseline (rank 0, N = 1 only)
     if rank == 0 and world == 1 and not args.no_cpu:
-        result["cpu_baseline"] = cpu_baseline(cfg, off, budget_s=args.cpu_seconds)
+        result["cpu_baseline"], result["parity"] = cpu_baseline(cfg, off, budget_s=args.cpu_seconds, gpu=gpu_prompt0)
     ctx.close()
     if rank == 0:
         print(json.dumps(result))
@@ -298,6 +318,37 @@ def run_ours(args):
         import torch.distributed as dist
         dist.barrier()
         dist.destroy_process_group()
+
+
+def sustained_leg(skv, ctx, step, ms_step, cfg, ab, peak, tiles_per_sm, world, dev, local) -> dict:
+    """Repeats the step back to back for about SUSTAIN_SECONDS (at least 600 steps) with the clocks
+    sampled every 50 ms; stage times are those of the last 64 steps."""
+    n = int(min(4000, max(600, SUSTAIN_SECONDS * 1e3 / ms_step)))
+    sampler = ClockSampler(local)
+    sampler.start()
+    barrier(world)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_begin = time.time()
+    e0.record()
+    for _ in range(n):
+        step()
+    e1.record()
+    barrier(world)
+    t_end = time.time()
+    clocks = sampler.stop(t_begin, t_end)
+    ms = max_over_ranks(e0.elapsed_time(e1), world, dev) / n
+    st = np.array([skv.shotkv_profile_read(ctx, i) for i in range(64)]).mean(axis=0)
+    mhz = clocks.get("sm_mhz") or 0.0
+    gbs = ab["total"] / (ms * 1e-3) / 1e9
+    return {"steps": n, "seconds": round(ms * n * 1e-3, 3), "ms_per_step": round(ms, 4),
+            "value": round(cfg.B * cfg.N * world / (ms * 1e-3), 1), "unit": UNIT,
+            "path_gbs": round(gbs, 1), "path_frac_of_measured_hbm": round(gbs / peak, 4),
+            "stage_ms": {"score": round(float(st[0]), 4), "shot_reduce": round(float(st[1]), 4),
+                         "select": round(float(st[2]), 4), "compact": round(float(st[3]), 4)},
+            "score_gbs": round(ab["k_read"] / (float(st[0]) * 1e-3) / 1e9, 1),
+            "score_frac_of_measured_hbm": round(ab["k_read"] / (float(st[0]) * 1e-3) / 1e9 / peak, 4),
+            "score_cycles_per_tile": round(float(st[0]) * 1e-3 * mhz * 1e6 / tiles_per_sm, 1) if mhz else None,
+            "clocks": clocks}
 
 
 def e2e_leg(skv, ctx, cfg, dims, pol, Q, K, V, off, Mcap, world, dev, args) -> dict:
@@ -425,7 +476,6 @@ def decode_leg(skv, ctx, rank, world, dev, peak, args) -> dict:
             "roofline": {"bound": "hbm", "kernel": "decode score kernel (last 64 steps)",
                          "achieved": round(per_step_bytes / (score_ms * 1e-3) / 1e9, 1), "peak": peak, "unit": "GB/s",
                          "frac": round(per_step_bytes / (score_ms * 1e-3) / 1e9 / peak, 4),
-                         # profiles/decode_score_kernel_cfg4_B2.md: dram read+write = 1.012 x algorithmic
                          "traffic": int(DECODE_TRAFFIC_RATIO * per_step_bytes) if DECODE_TRAFFIC_RATIO else None,
                          "algorithmic_bytes_per_launch": int(per_step_bytes), "ms_per_launch": round(score_ms, 4)},
             "path_frac_of_measured_hbm": round(per_step_bytes / (ms / dc.steps * 1e-3) / 1e9 / peak, 4),
@@ -442,27 +492,79 @@ def oracle_threads() -> int:
         return 1
 
 
-def oracle_unit_seconds(cfg, b, l, off_b) -> float:
+def oracle_unit_seconds(cfg, b, l, off_b, keep_result: bool = False):
     """Times the oracle, as it stands, on one (prompt, layer) unit of the workload."""
     from oracle import shotkv_oracle as O
     Q, K, V = wl.prefill_unit(cfg, b, l, off_b, "cpu")
     q, k, v = wl.bf16_to_f64(Q), wl.bf16_to_f64(K), wl.bf16_bits(V)
     t0 = time.perf_counter()
-    O.prefill_compress(q, k, v, off_b, cfg.r_p)
-    return time.perf_counter() - t0
+    ref = O.prefill_compress(q, k, v, off_b, cfg.r_p)
+    dt = time.perf_counter() - t0
+    if not keep_result:
+        return dt
+    ref["Kc_bits"] = O.compact_kv(wl.bf16_bits(K), ref["kept_idx"])
+    return dt, ref
 
 
-def cpu_baseline(cfg, off, budget_s: float = 20.0) -> dict:
+PARITY_ROW_UNITS = 4       # units whose compacted K/V rows are compared bit for bit in the parity record
+SCORE_RTOL, SCORE_ATOL = 2e-3, 1e-7
+
+
+def parity_of_unit(ref: dict, gpu: dict, l: int, rec: dict) -> None:
+    """Folds one (prompt 0, layer l) unit into the parity record: the oracle's result `ref` (just
+    computed for the CPU baseline) against what the timed GPU steps left for the same unit."""
+    S = len(ref["shot_scores"])
+    g_sc = gpu["shot_scores"][l, :S].numpy().astype(np.float64)
+    err = np.abs(g_sc - ref["shot_scores"]) / np.maximum(np.abs(ref["shot_scores"]), 1e-300)
+    rec["max_rel_score_err"] = max(rec["max_rel_score_err"], float(err.max()) if S else 0.0)
+    rec["scores_within_tol"] += int(np.all(np.abs(g_sc - ref["shot_scores"]) <= SCORE_RTOL * np.abs(ref["shot_scores"]) + SCORE_ATOL))
+    g_keep = gpu["keep"][l, :S].numpy()
+    n = int(gpu["kept_count"][l])
+    same = bool(np.array_equal(g_keep, ref["keep"]))
+    rec["units_checked"] += 1
+    if same:
+        rec["kept_sets_equal"] += 1
+        ok = n == len(ref["kept_idx"]) and np.array_equal(gpu["kept_idx"][l, :n].numpy(), ref["kept_idx"])
+        rec["kept_idx_equal"] += int(ok)
+        if l < gpu["Kc"].shape[0]:
+            rec["kv_rows_units"] += 1
+            rec["kv_rows_bit_exact"] += int(np.array_equal(wl.bf16_bits(gpu["Kc"][l, :, :n]), ref["Kc_bits"]) and
+                                            np.array_equal(wl.bf16_bits(gpu["Vc"][l, :, :n]), ref["Vc"]))
+    else:
+        # a tie: the kept sets differ; report how close the oracle's scores of the exchanged shots are
+        changed = np.nonzero(g_keep != ref["keep"])[0]
+        sc = ref["shot_scores"][changed]
+        gap = float((sc.max() - sc.min()) / max(abs(sc).max(), 1e-300)) if len(sc) else 0.0
+        rec["ties"] += 1
+        rec["closest_tie_rel_gap"] = gap if rec["closest_tie_rel_gap"] is None else min(rec["closest_tie_rel_gap"], gap)
+        rec["widest_tie_rel_gap"] = gap if rec["widest_tie_rel_gap"] is None else max(rec["widest_tie_rel_gap"], gap)
+        rec["tie_units"].append(int(l))
+        rec["ties_beyond_tolerance"] += int(gap > 2 * SCORE_RTOL)      # must stay 0: such a difference is an error, not a tie
+
+
+def cpu_baseline(cfg, off, budget_s: float = 20.0, gpu: dict | None = None):
     """The fp64 oracle on the host cores, on as many (prompt 0, layer l) units of the same workload
-    as fit in about `budget_s` seconds.  One unit = N tokens of one layer; a prompt is L units."""
+    as fit in about `budget_s` seconds.  One unit = N tokens of one layer; a prompt is L units.
+    With `gpu` (host copies of the timed steps' outputs for prompt 0) the oracle's results for those
+    units are also compared with them: returns (baseline, parity record)."""
+    rec = {"units_checked": 0, "sample": "", "score_tol": f"{SCORE_RTOL}*|ref| + {SCORE_ATOL}", "max_rel_score_err": 0.0,
+           "scores_within_tol": 0, "kept_sets_equal": 0, "kept_idx_equal": 0, "kv_rows_units": 0, "kv_rows_bit_exact": 0,
+           "ties": 0, "ties_beyond_tolerance": 0, "closest_tie_rel_gap": None, "widest_tie_rel_gap": None, "tie_units": []}
     t_total, n_units = 0.0, 0
     while t_total < budget_s and n_units < cfg.L:
-        t_total += oracle_unit_seconds(cfg, 0, n_units, off[0])
+        dt, ref = oracle_unit_seconds(cfg, 0, n_units, off[0], keep_result=True)
+        t_total += dt
+        if gpu is not None:
+            parity_of_unit(ref, gpu, n_units, rec)
         n_units += 1
     tokens_per_s = cfg.N / (t_total / n_units * cfg.L)
-    return {"value": round(tokens_per_s, 2), "unit": UNIT, "cores": oracle_threads(), "host_cpus": os.cpu_count(),
+    base = {"value": round(tokens_per_s, 2), "unit": UNIT, "cores": oracle_threads(), "host_cpus": os.cpu_count(),
             "kind": "oracle", "sample": f"{n_units} of {cfg.B * cfg.L} (prompt, layer) units of {cfg.name} "
                                         f"({n_units * cfg.N} token-layers) in {t_total:.1f} s; scaled to whole prompts"}
+    rec["sample"] = (f"prompt 0, layers 0..{n_units - 1} of the timed workload: the units the CPU baseline ran; a tie is a unit "
+                     "whose kept set differs from the oracle's (gap = spread of the oracle's scores over the exchanged shots)")
+    rec["max_rel_score_err"] = float(f"{rec['max_rel_score_err']:.3e}")
+    return base, (rec if gpu is not None else None)
 
 
 def run_reference(args):
@@ -515,6 +617,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the seconds-long repeat of the step")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

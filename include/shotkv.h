@@ -299,6 +299,29 @@ SHOTKV_API int shotkv_set_scoring_mode(shotkv_ctx* ctx, int mode);
  * over the calls finished so far on this context.  A diagnostic: 0 on ordinary inputs.  */
 SHOTKV_API uint64_t shotkv_repaired_items(const shotkv_ctx* ctx);
 
+/* Failure detection.  The tensor-core kernels of this library (the scoring pass of Section 5.1's
+ * prefill score equation and the per-token second pass) hand tiles between warps through shared-
+ * memory barriers.  Every such wait is bounded: after `cycles` SM clock cycles (default 4e9, about
+ * two seconds) the waiting warp gives up, raises its CTA's abort flag and a host-visible error
+ * word, all roles leave their loops, copies in flight are waited for (bounded again), tensor
+ * memory is released and the kernel returns.  The next call on the context then returns
+ * SHOTKV_ERR_TIMEOUT once (the outputs of the call that gave up are invalid); the call after
+ * that proceeds normally.  shotkv_set_wait_limit changes the limit for later launches of this
+ * context (0 restores the default).  */
+SHOTKV_API int shotkv_set_wait_limit(shotkv_ctx* ctx, int64_t cycles);
+/* Runs the bounded-wait helpers on purpose into their limit, so that the give-up path can be
+ * checked on any installation without disturbing a real kernel: one CTA, two barriers nobody
+ * arrives on.  Warp 0 waits as the epilogue warps do, with `limit_cycles` (1e3..1e9); one thread
+ * of warp 1 waits as the producer and MMA threads do, with four times that, and must leave early
+ * because warp 0 raised the abort flag.  Tensor memory is allocated and released around it as in
+ * the kernels' exit path.  Nothing faults and nothing spins past its limit.
+ *   report host [4] = {warp 0's wait succeeded (0 expected), warp 1's wait succeeded (0 expected),
+ *                      abort flag at exit (1 expected), cycles warp 1 waited (< 4*limit_cycles)}
+ * This call SYNCHRONISES `stream`.  It leaves the error word raised exactly as a real give-up
+ * does: the next call on the context returns SHOTKV_ERR_TIMEOUT, the one after that succeeds.  */
+SHOTKV_API int shotkv_selftest_bounded_wait(shotkv_ctx* ctx, int64_t limit_cycles, int32_t* report /* [4] */,
+                                            void* stream);
+
 /* Groups the single-pass form of shotkv_prefill_compress pipelines its units in: 0 (default)
  * chooses -- one group for device buffers, one per 256 MB of K (at most 4) for the host-buffer
  * variant, where the groups overlap uploads with write-backs --, 1 runs every step on the

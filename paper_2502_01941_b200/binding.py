@@ -34,6 +34,7 @@ EXPORTS = [
     "shotkv_decode_workspace_bytes", "shotkv_decode_capacity", "shotkv_decode_init", "shotkv_decode_step", "shotkv_decode_step_attend",
     "shotkv_profile_enable", "shotkv_profile_read", "shotkv_launch_count", "shotkv_select_shots_static", "shotkv_plan_pieces",
     "shotkv_set_scoring_mode", "shotkv_repaired_items", "shotkv_set_pipeline_groups",
+    "shotkv_set_wait_limit", "shotkv_selftest_bounded_wait",
 ]
 
 
@@ -101,6 +102,8 @@ def lib() -> C.CDLL:
         "shotkv_set_scoring_mode": (C.c_int, [vp, C.c_int]),
         "shotkv_set_pipeline_groups": (C.c_int, [vp, C.c_int]),
         "shotkv_repaired_items": (C.c_uint64, [vp]),
+        "shotkv_set_wait_limit": (C.c_int, [vp, C.c_int64]),
+        "shotkv_selftest_bounded_wait": (C.c_int, [vp, C.c_int64, C.POINTER(i32), vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(L, name)
@@ -359,6 +362,18 @@ def shotkv_set_scoring_mode(ctx: Context, mode: int) -> int:
 
 def shotkv_set_pipeline_groups(ctx: Context, groups: int) -> int:
     return ctx.check(lib().shotkv_set_pipeline_groups(ctx._h, int(groups)))
+
+
+def shotkv_set_wait_limit(ctx: Context, cycles: int) -> int:
+    return ctx.check(lib().shotkv_set_wait_limit(ctx._h, int(cycles)))
+
+
+def shotkv_selftest_bounded_wait(ctx: Context, limit_cycles: int, stream=None) -> list:
+    """Runs the bounded waits into their limit on a one-CTA kernel; returns the four report words.
+    Synchronises the stream and leaves the context's error word raised (see the header)."""
+    rep = (C.c_int32 * 4)()
+    ctx.check(lib().shotkv_selftest_bounded_wait(ctx._h, int(limit_cycles), rep, _stream(stream)))
+    return [int(rep[i]) for i in range(4)]
 
 
 def shotkv_repaired_items(ctx: Context) -> int:

@@ -61,15 +61,15 @@ __device__ __forceinline__ void mma_role_transposed(const Pipe<Cfg>& pp, const S
         if (nt <= 0) continue;
         if (u != cur_u) {
             if (cur_u >= 0) umma_commit(pp.qempty());
-            if (!(ok = mbar_wait_relaxed(pp.qfull(), qfphase, pp.abort_flag, p.err))) break;
+            if (!(ok = mbar_wait_relaxed(pp.qfull(), qfphase, pp.abort_flag, p.err, p.wait_cycles))) break;
             qfphase ^= 1;
             cur_u = u;
         }
         for (int t = 0; t < nt; ++t) {
             if (acc == which) {
-                if (!(ok = mbar_wait_relaxed(pp.full(stage), fphase, pp.abort_flag, p.err))) break;
+                if (!(ok = mbar_wait_relaxed(pp.full(stage), fphase, pp.abort_flag, p.err, p.wait_cycles))) break;
                 const uint32_t tph = acc ? tephase1 : tephase0;
-                if (!(ok = mbar_wait_relaxed(pp.tempty(acc, 0), tph, pp.abort_flag, p.err))) break;
+                if (!(ok = mbar_wait_relaxed(pp.tempty(acc, 0), tph, pp.abort_flag, p.err, p.wait_cycles))) break;
                 fence_after_sync();
                 const uint32_t kb = pp.sK + stage * Cfg::kStageBytes;
                 const uint32_t d_tmem = pp.tmem_base + (uint32_t)(acc * NR);
@@ -167,8 +167,8 @@ __global__ void __launch_bounds__(ColsumTcCfg<D, MB>::kThreads, 1)
             }
             for (int t = 0; t < nt; ++t) {
                 const uint32_t tph = acc ? tfphase1 : tfphase0;
-                if (!tc::mbar_try(pp.tfull(acc, 0), tph)) {
-                    bool w = lane == 0 ? tc::mbar_wait(pp.tfull(acc, 0), tph, pp.abort_flag, p.err) : true;
+                if (!__all_sync(0xffffffffu, tc::mbar_try(pp.tfull(acc, 0), tph))) {
+                    bool w = lane == 0 ? tc::mbar_wait(pp.tfull(acc, 0), tph, pp.abort_flag, p.err, p.wait_cycles) : true;
                     w = __shfl_sync(0xffffffffu, w, 0);
                     if (!w) ok = false;
                 }
@@ -229,7 +229,7 @@ __global__ void __launch_bounds__(ColsumTcCfg<D, MB>::kThreads, 1)
                 float* sl = slots + (quad * 2 + slot) * 32;
                 if (g == 1) {
                     if (ntile >= 2) {
-                        bool w = lane == 0 ? tc::mbar_wait(pp.extra_bar(bs + 1), par ^ 1u, pp.abort_flag, p.err) : true;
+                        bool w = lane == 0 ? tc::mbar_wait(pp.extra_bar(bs + 1), par ^ 1u, pp.abort_flag, p.err, p.wait_cycles) : true;
                         w = __shfl_sync(0xffffffffu, w, 0);
                         __syncwarp();
                         if (!w) ok = false;
@@ -238,7 +238,7 @@ __global__ void __launch_bounds__(ColsumTcCfg<D, MB>::kThreads, 1)
                     __syncwarp();
                     if (lane == 0) tc::mbar_arrive(pp.extra_bar(bs));
                 } else {
-                    bool w = lane == 0 ? tc::mbar_wait(pp.extra_bar(bs), par, pp.abort_flag, p.err) : true;
+                    bool w = lane == 0 ? tc::mbar_wait(pp.extra_bar(bs), par, pp.abort_flag, p.err, p.wait_cycles) : true;
                     w = __shfl_sync(0xffffffffu, w, 0);
                     __syncwarp();
                     if (!w) ok = false;

@@ -191,11 +191,17 @@ __global__ void __launch_bounds__(ScoreFastCfg<D, MB>::kThreads, 1)
                 }
                 const int slot = nflush & (RD - 1);
                 const uint32_t par = (uint32_t)(nflush / RD) & 1u;
+                // out of range (or not a number): the exact kernel redoes the item.  Tested on this
+                // slice's own sum, before any rescaling by another slice's reference could hide it.
+                if (live && !(zz < tc::kRedoAbove)) {
+                    p.redo[it] = 1;
+                    *p.redo_any = 1;
+                }
                 if (slice != 0) {
                     const int ring = (blk * 4 + quad) * (NSL - 1) + (slice - 1);
                     const int rs = ring * RD + slot;
                     if (nflush >= RD) {                                   // the slot's previous contents must have been read
-                        bool w = lane == 0 ? tc::mbar_wait(pp.extra_bar(rs * 2 + 1), par ^ 1u, pp.abort_flag, p.err) : true;
+                        bool w = lane == 0 ? tc::mbar_wait(pp.extra_bar(rs * 2 + 1), par ^ 1u, pp.abort_flag, p.err, p.wait_cycles) : true;
                         w = __shfl_sync(0xffffffffu, w, 0);
                         __syncwarp();
                         ok = ok && w;
@@ -209,7 +215,7 @@ __global__ void __launch_bounds__(ScoreFastCfg<D, MB>::kThreads, 1)
 #pragma unroll
                     for (int s = 1; s < NSL; ++s) {
                         const int rs = ((blk * 4 + quad) * (NSL - 1) + (s - 1)) * RD + slot;
-                        bool w = lane == 0 ? tc::mbar_wait(pp.extra_bar(rs * 2), par, pp.abort_flag, p.err) : true;
+                        bool w = lane == 0 ? tc::mbar_wait(pp.extra_bar(rs * 2), par, pp.abort_flag, p.err, p.wait_cycles) : true;
                         w = __shfl_sync(0xffffffffu, w, 0);
                         __syncwarp();                                     // orders the other lanes' reads after lane 0's wait
                         ok = ok && w;
@@ -227,10 +233,6 @@ __global__ void __launch_bounds__(ScoreFastCfg<D, MB>::kThreads, 1)
                     const size_t o = ((size_t)u * p.P + pi) * p.Rpad + row;
                     p.part_m[o] = live ? mm : 0.f;
                     p.part_z[o] = live ? zz : 0.f;
-                    if (live && !(zz < tc::kRedoAbove)) {  // out of range (or not a number): the exact kernel redoes the item
-                        p.redo[it] = 1;
-                        *p.redo_any = 1;
-                    }
                 }
                 z[0] = z[1] = 0ull;
                 ++nflush;
@@ -267,8 +269,9 @@ __global__ void __launch_bounds__(ScoreFastCfg<D, MB>::kThreads, 1)
 
             for (int t = 0; t < nt; ++t) {
                 const uint32_t tph = acc ? tfphase1 : tfphase0;
-                if (!tc::mbar_try(pp.tfull(acc, blk), tph)) {            // usually ready: one test by the whole warp
-                    bool w = lane == 0 ? tc::mbar_wait(pp.tfull(acc, blk), tph, pp.abort_flag, p.err) : true;   // one poller per warp
+                // usually ready: one test by the whole warp, made uniform before anything depends on it
+                if (!__all_sync(0xffffffffu, tc::mbar_try(pp.tfull(acc, blk), tph))) {
+                    bool w = lane == 0 ? tc::mbar_wait(pp.tfull(acc, blk), tph, pp.abort_flag, p.err, p.wait_cycles) : true;   // one poller per warp
                     w = __shfl_sync(0xffffffffu, w, 0);
                     if (!w) ok = false;
                 }

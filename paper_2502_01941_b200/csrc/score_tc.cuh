@@ -44,6 +44,7 @@ struct ScoreTcParams {
     float* part_m;        // [U][P][Rpad]
     float* part_z;        // [U][P][Rpad]
     int* err;             // error word (host-visible); set to 1 when a bounded wait gave up
+    long long wait_cycles;    // limit of every bounded wait, in SM clock cycles
     // Item filter.  The fast kernel (score_fast.cuh) raises redo[item] and *redo_any when an item's
     // sums left the fp32 range it works in; the exact kernel, given the same arrays, recomputes
     // only those items and returns at once when there is none.  Both NULL: every item is done.
@@ -69,7 +70,7 @@ struct ScoreTcCfg {
 namespace tc {
 
 constexpr int kTileKeys = 128;
-constexpr long long kWaitCycles = 4000000000LL;   // about two seconds
+constexpr long long kWaitCycles = 4000000000LL;   // default limit of a bounded wait: about two seconds
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
@@ -91,15 +92,17 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
         : "memory");
     return done != 0;
 }
-// Bounded wait.  Returns false when the CTA is aborting (this waiter gave up, or another did).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* err) {
+// Bounded wait: gives up after `limit` cycles.  Returns false when the CTA is aborting (this
+// waiter gave up, or another did); the waiter that gives up raises the CTA's abort flag and the
+// device error word.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* err, long long limit) {
     if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
     for (uint32_t spin = 1;; ++spin) {
         if (mbar_try(bar, parity)) return true;
         if ((spin & 63u) == 0u) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitCycles) {
+            if (clock64() - t0 > limit) {
                 *abort_flag = 1;
                 atomicExch(err, 1);
                 return false;
@@ -110,7 +113,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 
 // The same for the single-thread producer and MMA roles, which wait long and often: sleeping
 // between polls keeps their spinning out of the issue slots the epilogue warps need.
-__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* err) {
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* err, long long limit) {
     if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
     for (uint32_t spin = 1;; ++spin) {
@@ -118,7 +121,7 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity,
         if (mbar_try(bar, parity)) return true;
         if ((spin & 15u) == 0u) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitCycles) {
+            if (clock64() - t0 > limit) {
                 *abort_flag = 1;
                 atomicExch(err, 1);
                 return false;
@@ -372,7 +375,7 @@ __device__ __forceinline__ void producer_role(const Pipe<Cfg>& pp, const CUtenso
         const int nt = (hi - lo + TN - 1) / TN;
         if (nt <= 0) continue;
         if (u != cur_u) {
-            if (!(ok = mbar_wait_relaxed(pp.qempty(), qephase, pp.abort_flag, p.err))) break;
+            if (!(ok = mbar_wait_relaxed(pp.qempty(), qephase, pp.abort_flag, p.err, p.wait_cycles))) break;
             qephase ^= 1;
             mbar_expect_tx(pp.qfull(), MB * NSUB * q_box_rows * 128);
 #pragma unroll
@@ -384,7 +387,7 @@ __device__ __forceinline__ void producer_role(const Pipe<Cfg>& pp, const CUtenso
             cur_u = u;
         }
         for (int t = 0; t < nt; ++t) {
-            if (!(ok = mbar_wait_relaxed(pp.empty(stage), ephase, pp.abort_flag, p.err))) break;
+            if (!(ok = mbar_wait_relaxed(pp.empty(stage), ephase, pp.abort_flag, p.err, p.wait_cycles))) break;
             mbar_expect_tx(pp.full(stage), NSUB * k_box_rows * 128);
 #pragma unroll
             for (int sub = 0; sub < NSUB; ++sub)
@@ -406,7 +409,7 @@ __device__ __forceinline__ void producer_role(const Pipe<Cfg>& pp, const CUtenso
                 s = NST - 1;
                 ph ^= 1;
             }
-            while (!mbar_try(pp.full(s), ph ^ 1) && clock64() - t0 < kWaitCycles) {
+            while (!mbar_try(pp.full(s), ph ^ 1) && clock64() - t0 < p.wait_cycles) {
             }
         }
     }
@@ -435,19 +438,19 @@ __device__ __forceinline__ void mma_role(const Pipe<Cfg>& pp, const ScoreTcParam
         if (nt <= 0) continue;
         if (u != cur_u) {
             if (cur_u >= 0) umma_commit(pp.qempty());     // Q may be replaced once these MMAs are done
-            if (!(ok = mbar_wait_relaxed(pp.qfull(), qfphase, pp.abort_flag, p.err))) break;
+            if (!(ok = mbar_wait_relaxed(pp.qfull(), qfphase, pp.abort_flag, p.err, p.wait_cycles))) break;
             qfphase ^= 1;
             cur_u = u;
         }
         for (int t = 0; t < nt; ++t) {
             const bool mine = NT == 1 || acc == which;
             if (mine) {
-            if (!(ok = mbar_wait_relaxed(pp.full(stage), fphase, pp.abort_flag, p.err))) break;
+            if (!(ok = mbar_wait_relaxed(pp.full(stage), fphase, pp.abort_flag, p.err, p.wait_cycles))) break;
             const uint32_t tph = acc ? tephase1 : tephase0;
             const uint32_t kb = pp.sK + stage * Cfg::kStageBytes;
 #pragma unroll
             for (int b = 0; b < MB; ++b) {
-                if (!(ok = mbar_wait_relaxed(pp.tempty(acc, b), tph, pp.abort_flag, p.err))) break;
+                if (!(ok = mbar_wait_relaxed(pp.tempty(acc, b), tph, pp.abort_flag, p.err, p.wait_cycles))) break;
                 fence_after_sync();
                 const uint32_t d_tmem = pp.tmem_base + (uint32_t)((acc * MB + b) * TN);
 #pragma unroll
@@ -597,7 +600,7 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
 
             for (int t = 0; t < nt; ++t) {
                 const uint32_t tph = acc ? tfphase1 : tfphase0;
-                ok = lane == 0 ? tc::mbar_wait(bar_tfull(acc, blk), tph, abort_flag, p.err) : true;   // one poller per warp
+                ok = lane == 0 ? tc::mbar_wait(bar_tfull(acc, blk), tph, abort_flag, p.err, p.wait_cycles) : true;   // one poller per warp
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) break;
                 if (acc) tfphase1 ^= 1; else tfphase0 ^= 1;
@@ -640,6 +643,57 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
         __syncwarp();
         tc::fence_after_sync();
         tc::tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// Self-test of the bounded waits, for the host to run on demand: one CTA, two warps, two mbarriers
+// that nobody ever arrives on.  Warp 0 waits on the first the way the epilogue warps do (lane 0
+// polls with mbar_wait, the result is shuffled to the warp) with the given limit; lane 0 of warp 1
+// waits on the second the way the producer and MMA threads do (mbar_wait_relaxed) with four times
+// the limit, so it must leave because warp 0 raised the abort flag, not because its own time ran
+// out.  Tensor memory is allocated at the start and released at the end, as in the kernels' exit
+// path after an abort.  report[0..3] = {warp 0's wait returned true, warp 1's wait returned true,
+// abort flag at exit, cycles warp 1 waited (saturated at 2^31 - 1)}.  The error word is raised
+// exactly as in a real give-up, so the next call on the context reports it.
+__global__ void __launch_bounds__(64, 1) bounded_wait_selftest_kernel(long long limit, int* err, int* report) {
+    __shared__ __align__(8) unsigned long long bars[2];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_word;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t bar0 = smem_u32(&bars[0]), bar1 = smem_u32(&bars[1]);
+    volatile int* abort_flag = &abort_word;
+    if (threadIdx.x == 0) {
+        tc::mbar_init(bar0, 1);
+        tc::mbar_init(bar1, 1);
+        abort_word = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        tc::tmem_alloc(smem_u32(&tmem_slot), 32);
+        tc::tmem_relinquish();
+    }
+    tc::fence_before_sync();
+    __syncthreads();
+    tc::fence_after_sync();
+    const uint32_t tmem_base = tmem_slot;
+    if (warp == 0) {
+        bool ok = lane == 0 ? tc::mbar_wait(bar0, 0, abort_flag, err, limit) : true;
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (lane == 0) report[0] = ok ? 1 : 0;
+    } else if (lane == 0) {
+        const long long t0 = clock64();
+        const bool ok = tc::mbar_wait_relaxed(bar1, 0, abort_flag, err, 4 * limit);
+        const long long dt = clock64() - t0;
+        report[1] = ok ? 1 : 0;
+        report[3] = dt > 0x7fffffffLL ? 0x7fffffff : (int)dt;
+    }
+    tc::fence_before_sync();
+    __syncthreads();
+    if (threadIdx.x == 0) report[2] = *abort_flag;
+    if (warp == 0) {
+        __syncwarp();
+        tc::fence_after_sync();
+        tc::tmem_dealloc(tmem_base, 32);
     }
 }
 

@@ -32,6 +32,8 @@ constexpr size_t kStageSlotBytes = 1u << 20;
 constexpr int kProfSlots = 64;
 constexpr int kMaxGroups = 4;         // most groups the fused prefill call pipelines its units in
 constexpr double kMinGroupKBytes = 256.0 * 1024 * 1024;   // least K a group of the automatic split holds
+constexpr int kErrWords = 8;           // ints of host-mapped memory the kernels report through
+constexpr int kBigSmem = 200 * 1024;   // dynamic shared memory the small kernels are allowed (set once per context)
 
 inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
@@ -65,6 +67,9 @@ struct shotkv_ctx {
     int* err_dev = nullptr;
     int sm_count = 148;
     int scoring_mode = SHOTKV_SCORING_FAST;
+    long long wait_cycles = tc::kWaitCycles;   // limit of every bounded device-side wait
+    int32_t* static_offsets = nullptr;         // device address of the built-in boundary table (looked up on first use)
+    void* encode_tiled = nullptr;              // cuTensorMapEncodeTiled, resolved at creation
 };
 
 namespace {
@@ -206,19 +211,19 @@ PrefillWs carve(const shotkv_dims* d, void* base) {
 // Copies `bytes` of host data to `dst` on `stream` through the context's pinned ring, so the
 // caller's buffer may be reused at once and the host does not wait for the stream.
 int upload_small(shotkv_ctx* ctx, void* dst, const void* src, size_t bytes, cudaStream_t stream) {
-    if (bytes == 0) return SHOTKV_OK;
-    if (bytes > kStageSlotBytes) {
-        CUDA_TRY(ctx, cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, stream));
-        CUDA_TRY(ctx, cudaStreamSynchronize(stream));
-        return SHOTKV_OK;
+    // one ring slot at a time; a table larger than a slot goes in several copies.  The host waits
+    // only for the copy that last used the slot it is about to refill, never for the stream.
+    for (size_t done = 0; done < bytes;) {
+        const size_t n = bytes - done < kStageSlotBytes ? bytes - done : kStageSlotBytes;
+        const int slot = ctx->stage_next;
+        ctx->stage_next = (slot + 1) % kStageSlots;
+        CUDA_TRY(ctx, cudaEventSynchronize(ctx->stage_done[slot]));
+        unsigned char* s = ctx->stage + (size_t)slot * kStageSlotBytes;
+        memcpy(s, (const unsigned char*)src + done, n);
+        CUDA_TRY(ctx, cudaMemcpyAsync((unsigned char*)dst + done, s, n, cudaMemcpyHostToDevice, stream));
+        CUDA_TRY(ctx, cudaEventRecord(ctx->stage_done[slot], stream));
+        done += n;
     }
-    const int slot = ctx->stage_next;
-    ctx->stage_next = (slot + 1) % kStageSlots;
-    CUDA_TRY(ctx, cudaEventSynchronize(ctx->stage_done[slot]));
-    unsigned char* s = ctx->stage + (size_t)slot * kStageSlotBytes;
-    memcpy(s, src, bytes);
-    CUDA_TRY(ctx, cudaMemcpyAsync(dst, s, bytes, cudaMemcpyHostToDevice, stream));
-    CUDA_TRY(ctx, cudaEventRecord(ctx->stage_done[slot], stream));
     return SHOTKV_OK;
 }
 
@@ -309,23 +314,20 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-EncodeTiledFn encode_tiled_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = (EncodeTiledFn)p;
-    }
-    return fn;
+// Resolved once per context, at creation (no process-wide state).
+void* resolve_encode_tiled() {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+        return p;
+    return nullptr;
 }
 
 template <int D, int MB>
 int launch_score_tc_t(shotkv_ctx* ctx, const CUtensorMap& tmQ, const CUtensorMap& tmK, int qbox, int kbox,
                       const ScoreTcParams& sp, cudaStream_t stream) {
     constexpr int smem = ScoreTcCfg<D, MB>::kSmemBytes;
-    CUDA_TRY(ctx, cudaFuncSetAttribute(score_tc_kernel<D, MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     int grid = sp.total_items < ctx->sm_count ? sp.total_items : ctx->sm_count;
     if (grid < 1) grid = 1;
     score_tc_kernel<D, MB><<<grid, ScoreTcCfg<D, MB>::kThreads, smem, stream>>>(tmQ, tmK, qbox, kbox, sp);
@@ -340,7 +342,6 @@ template <int D, int MB>
 int launch_score_fast_t(shotkv_ctx* ctx, const CUtensorMap& tmQ, const CUtensorMap& tmK, int qbox, int kbox,
                         const ScoreTcParams& sp, cudaStream_t stream) {
     constexpr int smem = ScoreFastCfg<D, MB>::kSmemBytes;
-    CUDA_TRY(ctx, cudaFuncSetAttribute(score_fast_kernel<D, MB, kPolyEvery>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     int grid = sp.total_items < ctx->sm_count ? sp.total_items : ctx->sm_count;
     if (grid < 1) grid = 1;
     score_fast_kernel<D, MB, kPolyEvery><<<grid, ScoreFastCfg<D, MB>::kThreads, smem, stream>>>(tmQ, tmK, qbox, kbox, sp);
@@ -357,7 +358,7 @@ struct TcSetup {
 };
 int tc_setup(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const shotkv_bf16* K, const PrefillWs& w, int P,
              const ChunkPlan& plan, TcSetup& t) {
-    EncodeTiledFn enc = encode_tiled_fn();
+    EncodeTiledFn enc = (EncodeTiledFn)ctx->encode_tiled;
     if (!enc) return fail(ctx, SHOTKV_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
     if (((uintptr_t)Q | (uintptr_t)K) & 15) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "Qwin and K must be 16-byte aligned");
     const long long U = (long long)d->B * d->L * d->Hkv;
@@ -395,6 +396,7 @@ int tc_setup(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const 
     sp.scale_log2 = kLog2e / sqrtf((float)d->d);
     sp.part_m = w.part_m; sp.part_z = w.part_z;
     sp.err = ctx->err_dev;
+    sp.wait_cycles = ctx->wait_cycles;
     sp.repaired = ctx->err_dev + 1;
     return SHOTKV_OK;
 }
@@ -402,7 +404,6 @@ int tc_setup(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const 
 template <int D, int MB>
 int launch_colsum_tc_t(shotkv_ctx* ctx, const TcSetup& t, const ColsumTcParams& cp, cudaStream_t stream) {
     constexpr int smem = ColsumTcCfg<D, MB>::kSmemBytes;
-    CUDA_TRY(ctx, cudaFuncSetAttribute(colsum_tc_kernel<D, MB, kPolyEvery>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     int grid = cp.base.total_items < ctx->sm_count ? cp.base.total_items : ctx->sm_count;
     if (grid < 1) grid = 1;
     colsum_tc_kernel<D, MB, kPolyEvery><<<grid, ColsumTcCfg<D, MB>::kThreads, smem, stream>>>(t.tmQ, t.tmK, t.qbox, t.kbox, cp);
@@ -562,11 +563,6 @@ PrefillWs group_ws(const PrefillWs& w, const shotkv_dims* d, const GroupView& v,
 int run_select(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_policy* p, const PrefillWs& w, float* shot_scores,
                uint8_t* keep, int32_t* kept_idx, int32_t* kept_count, int32_t Mcap, cudaStream_t stream) {
     const size_t smem = (size_t)d->S * 16 + (kSelectThreads + 1) * 4 + 16;
-    static bool attr_done = false;
-    if (smem > 48 * 1024 || !attr_done) {
-        CUDA_TRY(ctx, cudaFuncSetAttribute(select_shots_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
-        attr_done = true;
-    }
     select_shots_kernel<<<d->B * d->L, kSelectThreads, smem, stream>>>(shot_scores, w.off, d->L, d->N, d->S, budget_of(d, p),
                                                                      p->select_mode, Mcap, keep, kept_idx, kept_count);
     LAUNCH_CHECK(ctx);
@@ -586,6 +582,33 @@ int run_compact(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* K, con
         compact_kv_kernel<64><<<grid, 256, 0, stream>>>((const uint4*)K, (const uint4*)V, kept_idx, kept_count, d->Hkv, d->N, Mcap, (uint4*)Kc, (uint4*)Vc);
     LAUNCH_CHECK(ctx);
     return SHOTKV_OK;
+}
+
+// Dynamic shared-memory limits of every kernel that may need more than the 48 KB default.  A
+// function attribute belongs to the device's context, so it is set once when a shotkv_ctx is
+// created on that device, never on a launch path.
+template <int D, int MB>
+cudaError_t set_tc_attributes() {
+    cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<D, MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, ScoreTcCfg<D, MB>::kSmemBytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(score_fast_kernel<D, MB, kPolyEvery>, cudaFuncAttributeMaxDynamicSharedMemorySize, ScoreFastCfg<D, MB>::kSmemBytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(colsum_tc_kernel<D, MB, kPolyEvery>, cudaFuncAttributeMaxDynamicSharedMemorySize, ColsumTcCfg<D, MB>::kSmemBytes);
+    return e;
+}
+cudaError_t set_kernel_attributes() {
+    cudaError_t e = set_tc_attributes<128, 1>();
+    if (e == cudaSuccess) e = set_tc_attributes<128, 2>();
+    if (e == cudaSuccess) e = set_tc_attributes<64, 1>();
+    if (e == cudaSuccess) e = set_tc_attributes<64, 2>();
+    const void* small[] = {(const void*)select_shots_kernel, (const void*)shot_mass_kernel<128>, (const void*)shot_mass_kernel<256>,
+                           (const void*)decode_score_kernel<128>, (const void*)decode_score_kernel<64>,
+                           (const void*)decode_attend_kernel<128, 4>, (const void*)decode_attend_kernel<128, 8>,
+                           (const void*)decode_attend_kernel<64, 4>, (const void*)decode_attend_kernel<64, 8>,
+                           (const void*)decode_rank_kernel};
+    for (const void* f : small)
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kBigSmem);
+    return e;
 }
 
 }  // namespace
@@ -617,7 +640,7 @@ int shotkv_create(shotkv_ctx** out, int device) {
             delete ctx;
             return SHOTKV_ERR_CUDA;
         }
-    if (cudaHostAlloc((void**)&ctx->err_host, 2 * sizeof(int), cudaHostAllocMapped) != cudaSuccess ||
+    if (cudaHostAlloc((void**)&ctx->err_host, kErrWords * sizeof(int), cudaHostAllocMapped) != cudaSuccess ||
         cudaHostGetDevicePointer((void**)&ctx->err_dev, ctx->err_host, 0) != cudaSuccess) {
         shotkv_destroy(ctx);
         return SHOTKV_ERR_CUDA;
@@ -629,9 +652,14 @@ int shotkv_create(shotkv_ctx** out, int device) {
         shotkv_destroy(ctx);
         return SHOTKV_ERR_CUDA;
     }
-    ctx->err_host[0] = 0;      // word 0: a bounded wait gave up
-    ctx->err_host[1] = 0;      // word 1: work items the exact scoring kernel recomputed after the fast one
+    for (int i = 0; i < kErrWords; ++i) ctx->err_host[i] = 0;   // word 0: a bounded wait gave up; word 1: work items the
+                                                                 // exact scoring kernel recomputed; words 2-5: self-test report
     ctx->sm_count = prop.multiProcessorCount;
+    ctx->encode_tiled = resolve_encode_tiled();
+    if (set_kernel_attributes() != cudaSuccess) {
+        shotkv_destroy(ctx);
+        return SHOTKV_ERR_CUDA;
+    }
     *out = ctx;
     return SHOTKV_OK;
 }
@@ -754,17 +782,16 @@ static __device__ __align__(256) int32_t g_static_offsets[SHOTKV_STATIC_OFFSETS_
 namespace {
 // In host code `g_static_offsets` is only a handle; the address kernels can use has to be asked
 // for, per device, with that device current.
+// The address is kept in the context (a context belongs to one device), so nothing process-wide is
+// written: the first call of each context looks it up, with the context's device current.
 int static_offsets_ptr(shotkv_ctx* ctx, int32_t** out) {
-    static int32_t* ptr_of_device[64] = {};
-    const int dev = ctx->device;
-    if (dev < 0 || dev >= 64) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "device index %d beyond 63", dev);
-    if (!ptr_of_device[dev]) {
+    if (!ctx->static_offsets) {
         int32_t* p = nullptr;
         CUDA_TRY(ctx, cudaGetSymbolAddress((void**)&p, g_static_offsets));
         if (!p) return fail(ctx, SHOTKV_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
-        ptr_of_device[dev] = p;
+        ctx->static_offsets = p;
     }
-    *out = ptr_of_device[dev];
+    *out = ctx->static_offsets;
     return SHOTKV_OK;
 }
 }  // namespace
@@ -876,15 +903,18 @@ int prefill_compress_impl(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv
     if ((rc = prepare_pieces(ctx, dims, offsets_host, plan, w, &P, stream))) return rc;
     const size_t msm = (size_t)P * (Rpad / 32 + 1) * 4;
     if (S > 0) {
-        if (msm > 200 * 1024) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "too many shots for the single-pass path (S = %d)", S);
-        if (msm > 48 * 1024) {
-            if (Rpad == 128) CUDA_TRY(ctx, cudaFuncSetAttribute(shot_mass_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)msm));
-            else CUDA_TRY(ctx, cudaFuncSetAttribute(shot_mass_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)msm));
-        }
+        if (msm > kBigSmem) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "too many shots for the single-pass path (S = %d)", S);
     }
     prof_begin(ctx);
     const bool forked = gs.n > 1;
     cudaStream_t tail = forked ? ctx->aux : stream;
+    // Once a group has been handed to the second stream, an early return must still order that
+    // work before whatever the caller enqueues next on `stream`.
+    bool handed = false;
+    auto bail = [&](int code) {
+        if (forked && handed && cudaEventRecord(ctx->ev_join, tail) == cudaSuccess) cudaStreamWaitEvent(stream, ctx->ev_join, 0);
+        return code;
+    };
     for (int g = 0; g < gs.n; ++g) {
         const GroupView v = group_view(dims, gs, g);
         const PrefillWs wg = group_ws(w, dims, v, g, P);
@@ -895,13 +925,14 @@ int prefill_compress_impl(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv
         float* scores_g = shot_scores + v.bl0 * S1;
         int32_t* idx_g = kept_idx + v.bl0 * (size_t)Mcap;
         int32_t* count_g = kept_count + v.bl0;
-        if (before_group && (rc = (*before_group)(v, stream))) return rc;
+        if (before_group && (rc = (*before_group)(v, stream))) return bail(rc);
         prof_gmark(ctx, g, 0, stream);
-        if ((rc = launch_score_tc(ctx, dg, Qwin + v.bl0 * dims->H * dims->W * row, Kg, wg, P, plan, stream))) return rc;
+        if ((rc = launch_score_tc(ctx, dg, Qwin + v.bl0 * dims->H * dims->W * row, Kg, wg, P, plan, stream))) return bail(rc);
         prof_gmark(ctx, g, 1, stream);
         if (forked) {
-            CUDA_TRY(ctx, cudaEventRecord(ctx->ev_fork[g], stream));
-            CUDA_TRY(ctx, cudaStreamWaitEvent(tail, ctx->ev_fork[g], 0));
+            if (cudaEventRecord(ctx->ev_fork[g], stream) != cudaSuccess || cudaStreamWaitEvent(tail, ctx->ev_fork[g], 0) != cudaSuccess)
+                return bail(fail(ctx, SHOTKV_ERR_CUDA, "could not hand a group of units to the second stream"));
+            handed = true;
         }
         prof_gmark(ctx, g, 2, tail);
         if (S > 0) {
@@ -909,14 +940,16 @@ int prefill_compress_impl(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv
                 shot_mass_kernel<128><<<Ug, 128, msm, tail>>>(wg.part_m, wg.part_z, wg.piece_seg, P, R, Rpad, dg->L, dg->Hkv, S, wg.unit_shot);
             else
                 shot_mass_kernel<256><<<Ug, 256, msm, tail>>>(wg.part_m, wg.part_z, wg.piece_seg, P, R, Rpad, dg->L, dg->Hkv, S, wg.unit_shot);
-            LAUNCH_CHECK(ctx);
+            ctx->launches += 1;
+            if (cudaGetLastError() != cudaSuccess) return bail(fail(ctx, SHOTKV_ERR_CUDA, "per-shot reduction failed to launch"));
             shot_score_from_mass_kernel<<<dg->B * dg->L, 128, 0, tail>>>(wg.unit_shot, wg.off, dg->L, dg->Hkv, S, scores_g);
-            LAUNCH_CHECK(ctx);
+            ctx->launches += 1;
+            if (cudaGetLastError() != cudaSuccess) return bail(fail(ctx, SHOTKV_ERR_CUDA, "per-shot score kernel failed to launch"));
         }
         prof_gmark(ctx, g, 3, tail);
-        if ((rc = run_select(ctx, dg, policy, wg, scores_g, keep + v.bl0 * S1, idx_g, count_g, Mcap, tail))) return rc;
+        if ((rc = run_select(ctx, dg, policy, wg, scores_g, keep + v.bl0 * S1, idx_g, count_g, Mcap, tail))) return bail(rc);
         prof_gmark(ctx, g, 4, tail);
-        if ((rc = run_compact(ctx, dg, Kg, Vg, idx_g, count_g, Mcap, Kc + v.u0 * (size_t)Mcap * row, Vc + v.u0 * (size_t)Mcap * row, tail))) return rc;
+        if ((rc = run_compact(ctx, dg, Kg, Vg, idx_g, count_g, Mcap, Kc + v.u0 * (size_t)Mcap * row, Vc + v.u0 * (size_t)Mcap * row, tail))) return bail(rc);
         prof_gmark(ctx, g, 5, tail);
     }
     if (forked) {
@@ -1094,8 +1127,7 @@ namespace {
 template <int D, int QR>
 int launch_decode_attend(shotkv_ctx* ctx, const DecodeParams& p, int U, cudaStream_t stream) {
     const size_t smem = ((size_t)8 * p.Dcap + 8 * 8 * 2 + 16 + 8 * 17 * 8 + (size_t)8 * QR * D) * 4;
-    CUDA_TRY(ctx, cudaFuncSetAttribute(decode_attend_kernel<D, QR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-    if (smem > 200 * 1024) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "Dcap too large for the attention-output step");
+    if (smem > kBigSmem) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "Dcap too large for the attention-output step");
     decode_attend_kernel<D, QR><<<U, 256, smem, stream>>>(p);
     return SHOTKV_OK;
 }
@@ -1132,10 +1164,8 @@ int decode_step_impl(shotkv_ctx* ctx, shotkv_decode_state* st, const shotkv_bf16
         else rc = small ? launch_decode_attend<64, 4>(ctx, p, U, stream) : launch_decode_attend<64, 8>(ctx, p, U, stream);
         if (rc) return rc;
     } else if (d.d == 128) {
-        CUDA_TRY(ctx, cudaFuncSetAttribute(decode_score_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
         decode_score_kernel<128><<<U, 256, smem, stream>>>(p);
     } else {
-        CUDA_TRY(ctx, cudaFuncSetAttribute(decode_score_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
         decode_score_kernel<64><<<U, 256, smem, stream>>>(p);
     }
     LAUNCH_CHECK(ctx);
@@ -1154,7 +1184,6 @@ int decode_step_impl(shotkv_ctx* ctx, shotkv_decode_state* st, const shotkv_bf16
         if (k > n) k = n;
         if (k < n) {
             const size_t rs = (size_t)n * 16 + (kSelectThreads + 1) * 4 + 16;
-            CUDA_TRY(ctx, cudaFuncSetAttribute(decode_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
             decode_rank_kernel<<<BL, kSelectThreads, rs, stream>>>(st->acc, st->born, st->Dcap, n, k,
                                                                    prot > 0 ? st->T - prot : 0x7fffffff, keep_pos);
             LAUNCH_CHECK(ctx);
@@ -1221,6 +1250,28 @@ int shotkv_set_scoring_mode(shotkv_ctx* ctx, int mode) {
     if (mode != SHOTKV_SCORING_FAST && mode != SHOTKV_SCORING_EXACT)
         return fail(ctx, SHOTKV_ERR_INVALID_ARG, "scoring mode must be SHOTKV_SCORING_FAST or SHOTKV_SCORING_EXACT");
     ctx->scoring_mode = mode;
+    return SHOTKV_OK;
+}
+
+int shotkv_set_wait_limit(shotkv_ctx* ctx, int64_t cycles) {
+    if (!ctx) return SHOTKV_ERR_INVALID_ARG;
+    if (cycles < 0) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "wait limit must be >= 0 cycles (0 restores the default)");
+    ctx->wait_cycles = cycles == 0 ? tc::kWaitCycles : (long long)cycles;
+    return SHOTKV_OK;
+}
+
+int shotkv_selftest_bounded_wait(shotkv_ctx* ctx, int64_t limit_cycles, int32_t* report, void* stream_) {
+    int rc = set_device(ctx);
+    if (rc) return rc;
+    if (!report) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "report must not be NULL");
+    if (limit_cycles < 1000 || limit_cycles > 1000000000LL)
+        return fail(ctx, SHOTKV_ERR_INVALID_ARG, "self-test limit must be between 1e3 and 1e9 cycles");
+    cudaStream_t stream = (cudaStream_t)stream_;
+    for (int i = 0; i < 4; ++i) ((volatile int*)ctx->err_host)[2 + i] = -1;
+    bounded_wait_selftest_kernel<<<1, 64, 0, stream>>>((long long)limit_cycles, ctx->err_dev, ctx->err_dev + 2);
+    LAUNCH_CHECK(ctx);
+    CUDA_TRY(ctx, cudaStreamSynchronize(stream));
+    for (int i = 0; i < 4; ++i) report[i] = ((volatile int*)ctx->err_host)[2 + i];
     return SHOTKV_OK;
 }
 

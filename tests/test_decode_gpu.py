@@ -65,8 +65,10 @@ def lockstep(ctx, cfg, M, units, counts=None, steps=None, attend=False, protect_
         orc[(b, l)] = O.DecodeOracle(wl.bf16_to_f64(Kc[b, l, :, :m]), cfg.H, cfg.r_d, cfg.recompress_every,
                                      Vc=wl.bf16_to_f64(Vc[b, l, :, :m]) if attend else None, protect_recent=protect_recent)
     ties = 0
+    max_n = 0
     for s in range(steps or cfg.steps):
         q, k, v = wl.decode_step_inputs(cfg, s, "cuda")
+        max_n = max(max_n, gpu.state.n_dec + 1)          # entries scored by this step, before any eviction
         gpu.step(q, k, v)
         torch.cuda.synchronize()
         n = gpu.state.n_dec
@@ -96,6 +98,9 @@ def lockstep(ctx, cfg, M, units, counts=None, steps=None, attend=False, protect_
                         assert abs(sc[j] - cut) <= 2 * (P.SCORE_RTOL * abs(cut) + P.SCORE_ATOL), \
                             f"step {s}: eviction differs beyond a tie"
                     ties += 1
+                    gaps = [abs(sc[j] - cut) / max(abs(cut), 1e-300) for j in diff]
+                    P.report_tie(f"decode unit (b={b}, l={l}) step {s}: survivors differ in entries born at "
+                                 f"{sorted(o.born[j] for j in diff)}", len(diff) // 2, min(gaps), max(gaps))
                     want = sorted(got)
                 o.apply_keep(want)
             assert o.n_dec == n and o.born == g_born[b, l, :n].tolist()
@@ -108,6 +113,7 @@ def lockstep(ctx, cfg, M, units, counts=None, steps=None, attend=False, protect_
                 np.testing.assert_array_equal(kd, np.stack(o.Kd, axis=1)) if n else None
                 vd = wl.bf16_bits(gpu.Vd[b, l, :, :n])
                 np.testing.assert_array_equal(vd, np.stack(o.Vd, axis=1)) if n else None
+    lockstep.largest_region = max(getattr(lockstep, "largest_region", 0), max_n)
     return ties
 
 
@@ -211,3 +217,28 @@ def test_decode_protected_recent_entries(ctx, protect):
     cfg = wl.DecodeConfig("dec_protect", B=2, L=1, H=8, Hkv=2, d=128, steps=40, r_d=0.25, recompress_every=8, cfg_id=27)
     ties = lockstep(ctx, cfg, 64, [(0, 0), (1, 0)], protect_recent=protect)
     assert ties <= 2
+
+
+@pytest.mark.parametrize("attend", [False, True], ids=["plain", "attend"])
+def test_decode_region_crosses_128_and_256_entries(ctx, attend):
+    """A slow eviction schedule (keep 90 %, every 64 steps) grows the decode region past 128, 256
+    and 384 entries within 448 steps: every loop of the decode kernels that strides over the
+    region by the block size takes a second and third trip, evictions rank more than 256
+    candidates, and the in-place compaction moves several 16-row passes."""
+    cfg = wl.DecodeConfig("dec_wide", B=2, L=2, H=8, Hkv=2, d=128, steps=448, r_d=0.9, recompress_every=64, cfg_id=28)
+    lockstep.largest_region = 0
+    ties = lockstep(ctx, cfg, 500, [(0, 0), (1, 1)], attend=attend)
+    assert lockstep.largest_region >= 384
+    assert ties <= 3
+
+
+@pytest.mark.parametrize("attend", [False, True], ids=["plain", "attend"])
+def test_decode_config4_all_1024_steps_two_units(ctx, attend):
+    """The decode benchmark's own run: config 4 for all of its 1,024 steps, so that the decode region
+    reaches its full 280 entries (evictions with n > 256) at the batch size that is timed; the oracle
+    follows two sampled (sequence, layer) units in lock-step."""
+    cfg = wl.DECODE_CONFIG
+    lockstep.largest_region = 0
+    ties = lockstep(ctx, cfg, 3276, [(1, 4), (6, 29)], attend=attend)
+    assert lockstep.largest_region >= 279
+    assert ties <= 6

@@ -8,6 +8,7 @@ import pytest
 import torch
 
 import paper_2502_01941_b200 as skv
+from oracle import shotkv_oracle as O
 from paper_2502_01941_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -26,17 +27,46 @@ def _run(ctx, cfg, r_p, mode, seed):
     # outputs for the workspace-free call are allocated before it; the call itself gets no workspace
     got = {k: torch.full_like(ref[k], 7) for k in ("shot_scores", "keep", "kept_idx", "kept_count")}
     torch.cuda.synchronize()
+    # the driver's own count of free device memory sees any allocation, whoever makes it (the
+    # framework's caching allocator only sees its own); nothing else allocates between the two
+    # readings.  The table's address is looked up once per context: warm that up first so the
+    # reading does not include the module being loaded.
+    if not getattr(ctx, "_static_warm", False):
+        skv.shotkv_select_shots_static(ctx, dims, pol, imp, off, got["shot_scores"], got["keep"], got["kept_idx"],
+                                       got["kept_count"], Mcap)
+        torch.cuda.synchronize()
+        ctx._static_warm = True
+        for k in got:
+            got[k].fill_(7)
+        torch.cuda.synchronize()
     before = torch.cuda.memory_allocated()
+    free_before, _ = torch.cuda.mem_get_info()
+    launches = skv.shotkv_launch_count(ctx)
     skv.shotkv_select_shots_static(ctx, dims, pol, imp, off, got["shot_scores"], got["keep"], got["kept_idx"],
                                    got["kept_count"], Mcap)
     torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, "device memory was allocated or freed during the call"
     assert torch.cuda.memory_allocated() == before
+    assert skv.shotkv_launch_count(ctx) - launches == 2          # per-shot scores, selection: kernels really ran
     # same kernels, same inputs: the scores agree within the tests' score tolerance (in fact bit
     # for bit) and every integer output is identical
     np.testing.assert_allclose(got["shot_scores"].cpu().numpy(), ref["shot_scores"].cpu().numpy(), rtol=2e-3, atol=1e-7)
     for k in ("keep", "kept_idx", "kept_count"):
         assert torch.equal(got[k], ref[k]), k
     assert int(got["kept_count"].min()) > 0
+    # and against the definition itself, not only the sibling call: scores from the oracle's
+    # per-shot mean of the same importances, the kept set from the oracle's selector fed the
+    # kernel's own float32 scores (both sides then decide in the kernel's precision)
+    for (b, l) in {(0, 0), (cfg.B - 1, cfg.L - 1)}:
+        want = O.shot_scores(imp[b, l].cpu().numpy().astype(np.float64), off[b])
+        g_sc = got["shot_scores"][b, l].cpu().numpy()
+        np.testing.assert_allclose(g_sc, want, rtol=2e-3, atol=1e-7)
+        keep, idx, _ = O.select_shots(g_sc, off[b], cfg.N, r_p, mode)
+        np.testing.assert_array_equal(got["keep"][b, l].cpu().numpy(), keep)
+        n = int(got["kept_count"][b, l])
+        assert n == len(idx)
+        np.testing.assert_array_equal(got["kept_idx"][b, l, :n].cpu().numpy(), idx)
 
 
 def test_static_selection_matches_workspace_form_twice_in_a_row():
