@@ -50,6 +50,7 @@ DECODE_TRAFFIC_RATIO = 1.012
 DECODE_ATTEND_TRAFFIC_RATIO = None
 NOMINAL_HBM_GBS = 8000.0
 SUSTAIN_SECONDS = 2.5           # length of the sustained repeat of the step
+SCORING_MODES = {"fast": 0, "exact": 1}
 
 
 # ------------------------------------------------------------------ small utilities
@@ -172,7 +173,7 @@ def run_ours(args):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     ctx = skv.Context(local)
-    skv.shotkv_set_scoring_mode(ctx, skv.SCORING_EXACT if args.scoring == "exact" else skv.SCORING_FAST)
+    skv.shotkv_set_scoring_mode(ctx, SCORING_MODES[args.scoring])
     skv.shotkv_set_pipeline_groups(ctx, args.groups)
     peak, peak_src = measured_peaks()
 
@@ -234,15 +235,20 @@ def run_ours(args):
     if not args.no_sustained:
         sustained = sustained_leg(skv, ctx, step, ms_step, cfg, ab, peak, tiles_per_sm, world, dev, local)
     # host copies of prompt 0's results, for the parity record taken beside the CPU baseline
-    gpu_prompt0 = {k: out[k][0].cpu() for k in ("shot_scores", "keep", "kept_idx", "kept_count")}
-    gpu_prompt0["Kc"] = out["Kc"][0, :PARITY_ROW_UNITS].cpu()
-    gpu_prompt0["Vc"] = out["Vc"][0, :PARITY_ROW_UNITS].cpu()
+    gpu_prompt0 = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        gpu_prompt0 = {k: out[k][0].cpu() for k in ("shot_scores", "keep", "kept_idx", "kept_count")}
+        gpu_prompt0["Kc"] = out["Kc"][0, :PARITY_ROW_UNITS].cpu()
+        gpu_prompt0["Vc"] = out["Vc"][0, :PARITY_ROW_UNITS].cpu()
+        # the very bytes the timed steps read: the oracle is given these, not a second draw
+        gpu_prompt0["Q"], gpu_prompt0["K"], gpu_prompt0["V"] = Q[0].cpu(), K[0].cpu(), V[0].cpu()
     # the per-clock rate is taken at the clock of the sustained region when there is one (tens of
     # samples), else at the clock sampled during the --steps region
-    sm_mhz = (sustained or {}).get("clocks", {}).get("sm_mhz") or clocks.get("sm_mhz") or 1965.0
+    sm_mhz = (sustained or {}).get("score_kernel_sm_mhz") or (sustained or {}).get("clocks", {}).get("sm_mhz") or clocks.get("sm_mhz") or 1965.0
     rate_ms = sustained["stage_ms"]["score"] if sustained else score_ms
     ex2_rate = logits / (rate_ms * 1e-3) / sm_count / (sm_mhz * 1e6)
-    kernel_name = ("score_fast_kernel" if args.scoring == "fast" else "score_tc_kernel") + \
+    fast_name = "score_stream_kernel" if cfg.G * cfg.W > 128 else "score_fast_kernel"
+    kernel_name = {"fast": fast_name, "exact": "score_tc_kernel"}[args.scoring] + \
         " (window QK^T on tcgen05 + softmax partials), one launch per step"
     roofline = {"bound": "hbm", "kernel": kernel_name,
                 "achieved": round(achieved, 1), "peak": peak, "peak_source": peak_src, "unit": "GB/s",
@@ -326,6 +332,7 @@ def sustained_leg(skv, ctx, step, ms_step, cfg, ab, peak, tiles_per_sm, world, d
     n = int(min(4000, max(600, SUSTAIN_SECONDS * 1e3 / ms_step)))
     sampler = ClockSampler(local)
     sampler.start()
+    skv.shotkv_profile_enable(ctx, True)
     barrier(world)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_begin = time.time()
@@ -338,7 +345,11 @@ def sustained_leg(skv, ctx, step, ms_step, cfg, ab, peak, tiles_per_sm, world, d
     clocks = sampler.stop(t_begin, t_end)
     ms = max_over_ranks(e0.elapsed_time(e1), world, dev) / n
     st = np.array([skv.shotkv_profile_read(ctx, i) for i in range(64)]).mean(axis=0)
-    mhz = clocks.get("sm_mhz") or 0.0
+    skv.shotkv_profile_enable(ctx, False)
+    # the scoring kernel's own clock: cycles and nanoseconds its first CTA ran for in the last launch
+    cyc, ns = skv.shotkv_last_scoring_clock(ctx)
+    kernel_mhz = cyc / ns * 1e3 if ns > 0 else None
+    mhz = kernel_mhz or clocks.get("sm_mhz") or 0.0
     gbs = ab["total"] / (ms * 1e-3) / 1e9
     return {"steps": n, "seconds": round(ms * n * 1e-3, 3), "ms_per_step": round(ms, 4),
             "value": round(cfg.B * cfg.N * world / (ms * 1e-3), 1), "unit": UNIT,
@@ -348,6 +359,7 @@ def sustained_leg(skv, ctx, step, ms_step, cfg, ab, peak, tiles_per_sm, world, d
             "score_gbs": round(ab["k_read"] / (float(st[0]) * 1e-3) / 1e9, 1),
             "score_frac_of_measured_hbm": round(ab["k_read"] / (float(st[0]) * 1e-3) / 1e9 / peak, 4),
             "score_cycles_per_tile": round(float(st[0]) * 1e-3 * mhz * 1e6 / tiles_per_sm, 1) if mhz else None,
+            "score_kernel_sm_mhz": round(kernel_mhz, 1) if kernel_mhz else None,
             "clocks": clocks}
 
 
@@ -492,10 +504,11 @@ def oracle_threads() -> int:
         return 1
 
 
-def oracle_unit_seconds(cfg, b, l, off_b, keep_result: bool = False):
-    """Times the oracle, as it stands, on one (prompt, layer) unit of the workload."""
+def oracle_unit_seconds(cfg, b, l, off_b, keep_result: bool = False, inputs=None):
+    """Times the oracle, as it stands, on one (prompt, layer) unit of the workload: on `inputs`
+    (Q, K, V of that unit as bf16 host tensors) when given, else on a draw of its own."""
     from oracle import shotkv_oracle as O
-    Q, K, V = wl.prefill_unit(cfg, b, l, off_b, "cpu")
+    Q, K, V = inputs if inputs is not None else wl.prefill_unit(cfg, b, l, off_b, "cpu")
     q, k, v = wl.bf16_to_f64(Q), wl.bf16_to_f64(K), wl.bf16_bits(V)
     t0 = time.perf_counter()
     ref = O.prefill_compress(q, k, v, off_b, cfg.r_p)
@@ -552,7 +565,8 @@ def cpu_baseline(cfg, off, budget_s: float = 20.0, gpu: dict | None = None):
            "ties": 0, "ties_beyond_tolerance": 0, "closest_tie_rel_gap": None, "widest_tie_rel_gap": None, "tie_units": []}
     t_total, n_units = 0.0, 0
     while t_total < budget_s and n_units < cfg.L:
-        dt, ref = oracle_unit_seconds(cfg, 0, n_units, off[0], keep_result=True)
+        ins = (gpu["Q"][n_units], gpu["K"][n_units], gpu["V"][n_units]) if gpu is not None else None
+        dt, ref = oracle_unit_seconds(cfg, 0, n_units, off[0], keep_result=True, inputs=ins)
         t_total += dt
         if gpu is not None:
             parity_of_unit(ref, gpu, n_units, rec)
@@ -609,7 +623,7 @@ def main():
     ap.add_argument("--units", default="shots", choices=["shots", "sentences", "chunks"],
                     help="semantic units of the timed workload: the config's few-shot examples (default), sentence-sized "
                          "units of 10-40 tokens (the document-QA adaptation), or fixed chunks of 16 tokens")
-    ap.add_argument("--scoring", default="fast", choices=["fast", "exact"],
+    ap.add_argument("--scoring", default="fast", choices=sorted(SCORING_MODES),
                     help="scoring kernel: the default pair (fast kernel + exact repair) or the exact kernel alone")
     ap.add_argument("--groups", type=int, default=0, choices=[0, 1, 2, 3, 4],
                     help="groups of units the fused call pipelines (0: the library's choice; 1: no overlap of steps)")

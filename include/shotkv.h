@@ -322,6 +322,13 @@ SHOTKV_API int shotkv_set_wait_limit(shotkv_ctx* ctx, int64_t cycles);
 SHOTKV_API int shotkv_selftest_bounded_wait(shotkv_ctx* ctx, int64_t limit_cycles, int32_t* report /* [4] */,
                                             void* stream);
 
+/* SM cycles and nanoseconds that the first CTA of the most recent scoring launch of this context
+ * ran for (its own cycle counter and the GPU's nanosecond timer, read at its start and end).  Their
+ * quotient is the SM clock the kernel really ran at -- under a power cap that is not the clock a
+ * sampler reads between kernels -- and cycles / tiles per SM is the kernel's cost per tile in the
+ * unit its arithmetic is counted in.  Valid once the launch has finished (synchronise first).  */
+SHOTKV_API int shotkv_last_scoring_clock(const shotkv_ctx* ctx, int64_t* cycles, int64_t* nanoseconds);
+
 /* Groups the single-pass form of shotkv_prefill_compress pipelines its units in: 0 (default)
  * chooses -- one group for device buffers, one per 256 MB of K (at most 4) for the host-buffer
  * variant, where the groups overlap uploads with write-backs --, 1 runs every step on the

@@ -34,7 +34,7 @@ EXPORTS = [
     "shotkv_decode_workspace_bytes", "shotkv_decode_capacity", "shotkv_decode_init", "shotkv_decode_step", "shotkv_decode_step_attend",
     "shotkv_profile_enable", "shotkv_profile_read", "shotkv_launch_count", "shotkv_select_shots_static", "shotkv_plan_pieces",
     "shotkv_set_scoring_mode", "shotkv_repaired_items", "shotkv_set_pipeline_groups",
-    "shotkv_set_wait_limit", "shotkv_selftest_bounded_wait",
+    "shotkv_set_wait_limit", "shotkv_selftest_bounded_wait", "shotkv_last_scoring_clock",
 ]
 
 
@@ -102,6 +102,7 @@ def lib() -> C.CDLL:
         "shotkv_set_scoring_mode": (C.c_int, [vp, C.c_int]),
         "shotkv_set_pipeline_groups": (C.c_int, [vp, C.c_int]),
         "shotkv_repaired_items": (C.c_uint64, [vp]),
+        "shotkv_last_scoring_clock": (C.c_int, [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
         "shotkv_set_wait_limit": (C.c_int, [vp, C.c_int64]),
         "shotkv_selftest_bounded_wait": (C.c_int, [vp, C.c_int64, C.POINTER(i32), vp]),
     }
@@ -374,6 +375,13 @@ def shotkv_selftest_bounded_wait(ctx: Context, limit_cycles: int, stream=None) -
     rep = (C.c_int32 * 4)()
     ctx.check(lib().shotkv_selftest_bounded_wait(ctx._h, int(limit_cycles), rep, _stream(stream)))
     return [int(rep[i]) for i in range(4)]
+
+
+def shotkv_last_scoring_clock(ctx: Context):
+    """(SM cycles, nanoseconds) of the first CTA of the latest scoring launch; synchronise first."""
+    c, n = C.c_int64(), C.c_int64()
+    ctx.check(lib().shotkv_last_scoring_clock(ctx._h, C.byref(c), C.byref(n)))
+    return int(c.value), int(n.value)
 
 
 def shotkv_repaired_items(ctx: Context) -> int:

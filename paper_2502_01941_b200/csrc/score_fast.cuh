@@ -133,6 +133,7 @@ __global__ void __launch_bounds__(ScoreFastCfg<D, MB>::kThreads, 1)
     constexpr int TN = tc::kTileKeys;
     constexpr int NSL = Cfg::kSlices, SLW = TN / NSL, NCH = SLW / 32, RD = Cfg::kRingDepth;
     extern __shared__ unsigned char smem_raw[];
+    tc::stamp(p.clk, 0);
     tc::Pipe<Cfg> pp;
     tc::pipe_setup(pp, smem_raw, Cfg::kEpiWarps / MB, Cfg::kRings * Cfg::kRingDepth * 2, 2);
     float* comb = tc::pipe_scratch(pp, smem_raw);     // [ring][slot][lane][m, z]
@@ -329,6 +330,7 @@ __global__ void __launch_bounds__(ScoreFastCfg<D, MB>::kThreads, 1)
 
     tc::fence_before_sync();
     __syncthreads();
+    tc::stamp(p.clk, 1);
     if (warp == 0) {
         __syncwarp();
         tc::fence_after_sync();

@@ -45,6 +45,7 @@ struct ScoreTcParams {
     float* part_z;        // [U][P][Rpad]
     int* err;             // error word (host-visible); set to 1 when a bounded wait gave up
     long long wait_cycles;    // limit of every bounded wait, in SM clock cycles
+    long long* clk;           // optional (host-visible): SM cycle counter and nanosecond timer of CTA 0 at kernel start and end
     // Item filter.  The fast kernel (score_fast.cuh) raises redo[item] and *redo_any when an item's
     // sums left the fp32 range it works in; the exact kernel, given the same arrays, recomputes
     // only those items and returns at once when there is none.  Both NULL: every item is done.
@@ -72,6 +73,17 @@ namespace tc {
 constexpr int kTileKeys = 128;
 constexpr long long kWaitCycles = 4000000000LL;   // default limit of a bounded wait: about two seconds
 
+// Diagnostic: CTA 0's SM cycle counter and the global nanosecond timer, written to clk[2*which] and
+// clk[2*which + 1] (which = 0 at kernel start, 1 at its end).  Their quotient is the SM clock the
+// kernel really ran at, which under a power cap is not the clock a sampler reads between kernels.
+__device__ __forceinline__ void stamp(long long* clk, int which) {
+    if (clk && blockIdx.x == 0 && threadIdx.x == 0) {
+        unsigned long long ns;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
+        clk[2 * which] = clock64();
+        clk[2 * which + 1] = (long long)ns;
+    }
+}
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
@@ -111,21 +123,33 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
-// The same for the single-thread producer and MMA roles, which wait long and often: sleeping
-// between polls keeps their spinning out of the issue slots the epilogue warps need.
+// try_wait that lets the hardware suspend the thread until the phase completes or about `ns`
+// nanoseconds have passed, whichever comes first.
+__device__ __forceinline__ bool mbar_try_suspend(uint32_t bar, uint32_t parity, uint32_t ns) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return done != 0;
+}
+// The same for the single-thread producer and MMA roles, which wait long and often.  They wait
+// suspended inside try_wait (up to a microsecond at a time) instead of polling: a polling loop with
+// short sleeps executed about 110 iterations per tile between the three of them, an eighth of all
+// the warp instructions of the kernel, in issue slots and power the epilogue warps need.
 __device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* err, long long limit) {
     if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
-    for (uint32_t spin = 1;; ++spin) {
-        __nanosleep(100);
-        if (mbar_try(bar, parity)) return true;
-        if ((spin & 15u) == 0u) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > limit) {
-                *abort_flag = 1;
-                atomicExch(err, 1);
-                return false;
-            }
+    for (;;) {
+        if (mbar_try_suspend(bar, parity, 1000u)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > limit) {
+            *abort_flag = 1;
+            atomicExch(err, 1);
+            return false;
         }
     }
 }
@@ -485,6 +509,7 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
     constexpr int NSL = Cfg::kSlices, SLW = TN / NSL, NCH = SLW / 32;     // slices, slice width, chunks per slice
     extern __shared__ unsigned char smem_raw[];
     if (p.redo_any && *p.redo_any == 0) return;       // repair launch with nothing to repair
+    tc::stamp(p.clk, 0);
     tc::Pipe<Cfg> pp;
     tc::pipe_setup(pp, smem_raw, 16 / MB);
     float* comb = tc::pipe_scratch(pp, smem_raw);     // [2][4][128][2]
@@ -639,6 +664,7 @@ __global__ void __launch_bounds__(ScoreTcCfg<D, MB>::kThreads, 1)
 
     tc::fence_before_sync();
     __syncthreads();
+    tc::stamp(p.clk, 1);
     if (warp == 0) {
         __syncwarp();
         tc::fence_after_sync();

@@ -17,6 +17,7 @@
 #include "common.cuh"
 #include "decode.cuh"
 #include "score_fast.cuh"
+#include "score_stream.cuh"
 #include "reductions.cuh"
 #include "score_tc.cuh"
 #include "select_compact.cuh"
@@ -32,7 +33,7 @@ constexpr size_t kStageSlotBytes = 1u << 20;
 constexpr int kProfSlots = 64;
 constexpr int kMaxGroups = 4;         // most groups the fused prefill call pipelines its units in
 constexpr double kMinGroupKBytes = 256.0 * 1024 * 1024;   // least K a group of the automatic split holds
-constexpr int kErrWords = 8;           // ints of host-mapped memory the kernels report through
+constexpr int kErrWords = 16;          // ints of host-mapped memory the kernels report through
 constexpr int kBigSmem = 200 * 1024;   // dynamic shared memory the small kernels are allowed (set once per context)
 
 inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
@@ -349,6 +350,17 @@ int launch_score_fast_t(shotkv_ctx* ctx, const CUtensorMap& tmQ, const CUtensorM
     return SHOTKV_OK;
 }
 
+template <int D>
+int launch_score_stream_t(shotkv_ctx* ctx, const CUtensorMap& tmQ, const CUtensorMap& tmK, int qbox, int kbox,
+                          const ScoreTcParams& sp, cudaStream_t stream) {
+    using Cfg = ScoreStreamCfg<D>;
+    int grid = sp.total_items < ctx->sm_count ? sp.total_items : ctx->sm_count;
+    if (grid < 1) grid = 1;
+    score_stream_kernel<D, kPolyEvery><<<grid, Cfg::kThreads, Cfg::kSmemBytes, stream>>>(tmQ, tmK, qbox, kbox, sp);
+    LAUNCH_CHECK(ctx);
+    return SHOTKV_OK;
+}
+
 // Tensor maps of Q (2-D: d x rows) and K (3-D: d x N x units), 64-element boxes with 128-byte swizzle, and the
 // parameters every tensor-core pass shares.
 struct TcSetup {
@@ -437,15 +449,17 @@ int launch_score_tc(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q,
     ScoreTcParams& sp = t.sp;
     const bool big = sp.Rpad == 256;
     int rc = SHOTKV_OK;
+    sp.clk = (long long*)(ctx->err_dev + 8);        // the first launch below stamps its clocks; a repair launch after it does not
     if (ctx->scoring_mode == SHOTKV_SCORING_FAST) {
         // fast kernel first; it marks the items whose sums left its range, and the exact kernel
         // below then redoes exactly those (returning at once when there is none)
         sp.redo_any = w.redo;
         sp.redo = w.redo + 1;
         CUDA_TRY(ctx, cudaMemsetAsync(w.redo, 0, ((size_t)sp.total_items + 1) * 4, stream));
-        if (d->d == 128) rc = big ? launch_score_fast_t<128, 2>(ctx, tmQ, tmK, qbox, kbox, sp, stream) : launch_score_fast_t<128, 1>(ctx, tmQ, tmK, qbox, kbox, sp, stream);
-        else rc = big ? launch_score_fast_t<64, 2>(ctx, tmQ, tmK, qbox, kbox, sp, stream) : launch_score_fast_t<64, 1>(ctx, tmQ, tmK, qbox, kbox, sp, stream);
+        if (d->d == 128) rc = big ? launch_score_stream_t<128>(ctx, tmQ, tmK, qbox, kbox, sp, stream) : launch_score_fast_t<128, 1>(ctx, tmQ, tmK, qbox, kbox, sp, stream);
+        else rc = big ? launch_score_stream_t<64>(ctx, tmQ, tmK, qbox, kbox, sp, stream) : launch_score_fast_t<64, 1>(ctx, tmQ, tmK, qbox, kbox, sp, stream);
         if (rc) return rc;
+        sp.clk = nullptr;
     }
     if (d->d == 128) return big ? launch_score_tc_t<128, 2>(ctx, tmQ, tmK, qbox, kbox, sp, stream) : launch_score_tc_t<128, 1>(ctx, tmQ, tmK, qbox, kbox, sp, stream);
     return big ? launch_score_tc_t<64, 2>(ctx, tmQ, tmK, qbox, kbox, sp, stream) : launch_score_tc_t<64, 1>(ctx, tmQ, tmK, qbox, kbox, sp, stream);
@@ -592,6 +606,8 @@ cudaError_t set_tc_attributes() {
     cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<D, MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, ScoreTcCfg<D, MB>::kSmemBytes);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(score_fast_kernel<D, MB, kPolyEvery>, cudaFuncAttributeMaxDynamicSharedMemorySize, ScoreFastCfg<D, MB>::kSmemBytes);
+    if (e == cudaSuccess && MB == 2)
+        e = cudaFuncSetAttribute(score_stream_kernel<D, kPolyEvery>, cudaFuncAttributeMaxDynamicSharedMemorySize, ScoreStreamCfg<D>::kSmemBytes);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(colsum_tc_kernel<D, MB, kPolyEvery>, cudaFuncAttributeMaxDynamicSharedMemorySize, ColsumTcCfg<D, MB>::kSmemBytes);
     return e;
@@ -653,7 +669,8 @@ int shotkv_create(shotkv_ctx** out, int device) {
         return SHOTKV_ERR_CUDA;
     }
     for (int i = 0; i < kErrWords; ++i) ctx->err_host[i] = 0;   // word 0: a bounded wait gave up; word 1: work items the
-                                                                 // exact scoring kernel recomputed; words 2-5: self-test report
+                                                                 // exact scoring kernel recomputed; words 2-5: self-test report;
+                                                                 // words 8-15: four 64-bit clock stamps of the last scoring launch
     ctx->sm_count = prop.multiProcessorCount;
     ctx->encode_tiled = resolve_encode_tiled();
     if (set_kernel_attributes() != cudaSuccess) {
@@ -1329,6 +1346,14 @@ int shotkv_profile_read(shotkv_ctx* ctx, int calls_back, float* stage_ms) {
 }
 
 uint64_t shotkv_launch_count(const shotkv_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int shotkv_last_scoring_clock(const shotkv_ctx* ctx, int64_t* cycles, int64_t* nanoseconds) {
+    if (!ctx || !ctx->err_host || !cycles || !nanoseconds) return SHOTKV_ERR_INVALID_ARG;
+    const volatile long long* w = (const volatile long long*)(ctx->err_host + 8);
+    *cycles = (int64_t)(w[2] - w[0]);
+    *nanoseconds = (int64_t)(w[3] - w[1]);
+    return SHOTKV_OK;
+}
 
 uint64_t shotkv_repaired_items(const shotkv_ctx* ctx) {
     return ctx && ctx->err_host ? (uint64_t)(unsigned)((volatile int*)ctx->err_host)[1] : 0;
