@@ -619,11 +619,14 @@ cudaError_t set_kernel_attributes() {
     if (e == cudaSuccess) e = set_tc_attributes<64, 2>();
     const void* small[] = {(const void*)select_shots_kernel, (const void*)shot_mass_kernel<128>, (const void*)shot_mass_kernel<256>,
                            (const void*)decode_score_kernel<128>, (const void*)decode_score_kernel<64>,
-                           (const void*)decode_attend_kernel<128, 4>, (const void*)decode_attend_kernel<128, 8>,
-                           (const void*)decode_attend_kernel<64, 4>, (const void*)decode_attend_kernel<64, 8>,
+                           (const void*)decode_attend_kernel<128>, (const void*)decode_attend_kernel<64>,
                            (const void*)decode_rank_kernel};
     for (const void* f : small)
         if (e == cudaSuccess) e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, kBigSmem);
+    // the fused decode step wants three CTAs of ~74 KB each on an SM: ask for the largest shared-memory carve-out
+    const void* wide[] = {(const void*)decode_attend_kernel<128>, (const void*)decode_attend_kernel<64>};
+    for (const void* f : wide)
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     return e;
 }
 
@@ -1141,11 +1144,12 @@ int shotkv_decode_init(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_po
 
 namespace {
 
-template <int D, int QR>
+template <int D>
 int launch_decode_attend(shotkv_ctx* ctx, const DecodeParams& p, int U, cudaStream_t stream) {
-    const size_t smem = ((size_t)8 * p.Dcap + 8 * 8 * 2 + 16 + 8 * 17 * 8 + (size_t)8 * QR * D) * 4;
+    using Cfg = AttendCfg<D>;
+    const size_t smem = ((size_t)8 * p.Dcap + Cfg::kWarps * 8 * 2 + 16) * 4 + Cfg::kRingBytes;
     if (smem > kBigSmem) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "Dcap too large for the attention-output step");
-    decode_attend_kernel<D, QR><<<U, 256, smem, stream>>>(p);
+    decode_attend_kernel<D><<<U, Cfg::kWarps * 32, smem, stream>>>(p);
     return SHOTKV_OK;
 }
 
@@ -1176,9 +1180,7 @@ int decode_step_impl(shotkv_ctx* ctx, shotkv_decode_state* st, const shotkv_bf16
     prof_begin(ctx);
     prof_mark(ctx, stream);
     if (attn_out) {
-        const bool small = p.G <= 4;
-        if (d.d == 128) rc = small ? launch_decode_attend<128, 4>(ctx, p, U, stream) : launch_decode_attend<128, 8>(ctx, p, U, stream);
-        else rc = small ? launch_decode_attend<64, 4>(ctx, p, U, stream) : launch_decode_attend<64, 8>(ctx, p, U, stream);
+        rc = d.d == 128 ? launch_decode_attend<128>(ctx, p, U, stream) : launch_decode_attend<64>(ctx, p, U, stream);
         if (rc) return rc;
     } else if (d.d == 128) {
         decode_score_kernel<128><<<U, 256, smem, stream>>>(p);
