@@ -45,9 +45,9 @@ FALLBACK_HBM_GBS = 6650.0
 # byte of the scoring kernel and of the two decode score kernels, taken on reduced copies of the
 # workloads (config 3 with B=1, L=8; config 4 with B=2) and scaled by the bytes of a full launch.
 # A ratio is set to None whenever its kernel has changed since its capture.
-SCORE_TC_TRAFFIC_RATIO = None
+SCORE_TC_TRAFFIC_RATIO = 1.043
 DECODE_TRAFFIC_RATIO = 1.012
-DECODE_ATTEND_TRAFFIC_RATIO = None
+DECODE_ATTEND_TRAFFIC_RATIO = 1.006
 NOMINAL_HBM_GBS = 8000.0
 SUSTAIN_SECONDS = 2.5           # length of the sustained repeat of the step
 SCORING_MODES = {"fast": 0, "exact": 1}
