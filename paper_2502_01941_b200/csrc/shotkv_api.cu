@@ -3,6 +3,7 @@
 #include "../../include/shotkv.h"
 
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <cmath>
 #include <cstdarg>
@@ -37,6 +38,16 @@ constexpr int kErrWords = 16;          // ints of host-mapped memory the kernels
 constexpr int kBigSmem = 200 * 1024;   // dynamic shared memory the small kernels are allowed (set once per context)
 
 inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+// Tracing: every compute entry point of the ABI is an NVTX range named after it, so that a
+// timeline tool shows which call enqueued which kernels.  NVTX is header-only and does nothing
+// unless a tool is attached to the process.
+struct TraceRange {
+    explicit TraceRange(const char* name) { nvtxRangePushA(name); }
+    ~TraceRange() { nvtxRangePop(); }
+    TraceRange(const TraceRange&) = delete;
+    TraceRange& operator=(const TraceRange&) = delete;
+};
 
 }  // namespace
 
@@ -752,6 +763,7 @@ size_t shotkv_workspace_bytes(const shotkv_dims* dims) {
 
 int shotkv_prefill_score(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_bf16* Qwin, const shotkv_bf16* K,
                          float* token_importance, void* ws, size_t ws_bytes, void* stream_) {
+    TraceRange trace_("shotkv_prefill_score");
     int rc = set_device(ctx);
     if (rc) return rc;
     const char* why = "";
@@ -768,6 +780,7 @@ int shotkv_prefill_score(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_
 int shotkv_select_shots(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_policy* policy,
                         const float* token_importance, const int32_t* offsets_host, float* shot_scores, uint8_t* keep,
                         int32_t* kept_idx, int32_t* kept_count, int32_t Mcap, void* ws, size_t ws_bytes, void* stream_) {
+    TraceRange trace_("shotkv_select_shots");
     int rc = set_device(ctx);
     if (rc) return rc;
     const char* why = "";
@@ -819,6 +832,7 @@ int static_offsets_ptr(shotkv_ctx* ctx, int32_t** out) {
 int shotkv_select_shots_static(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_policy* policy,
                                const float* token_importance, const int32_t* offsets_host, float* shot_scores,
                                uint8_t* keep, int32_t* kept_idx, int32_t* kept_count, int32_t Mcap, void* stream_) {
+    TraceRange trace_("shotkv_select_shots_static");
     int rc = set_device(ctx);
     if (rc) return rc;
     const char* why = "";
@@ -853,6 +867,7 @@ int shotkv_select_shots_static(shotkv_ctx* ctx, const shotkv_dims* dims, const s
 int shotkv_compact_kv(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv_bf16* K, const shotkv_bf16* V,
                       const int32_t* kept_idx, const int32_t* kept_count, int32_t Mcap, shotkv_bf16* Kc, shotkv_bf16* Vc,
                       void* stream_) {
+    TraceRange trace_("shotkv_compact_kv");
     int rc = set_device(ctx);
     if (rc) return rc;
     const char* why = "";
@@ -986,6 +1001,7 @@ int shotkv_prefill_compress(shotkv_ctx* ctx, const shotkv_dims* dims, const shot
                             uint8_t* keep, int32_t* kept_idx, int32_t* kept_count, int32_t Mcap, shotkv_bf16* Kc,
                             shotkv_bf16* Vc, float* token_importance, uint32_t flags, void* ws, size_t ws_bytes,
                             void* stream_) {
+    TraceRange trace_("shotkv_prefill_compress");
     return prefill_compress_impl(ctx, dims, policy, Qwin, K, V, offsets_host, shot_scores, keep, kept_idx, kept_count, Mcap, Kc,
                                  Vc, token_importance, flags, ws, ws_bytes, stream_, nullptr);
 }
@@ -1032,6 +1048,7 @@ int shotkv_prefill_compress_host(shotkv_ctx* ctx, const shotkv_dims* dims, const
                                  const int32_t* offsets_host, float* shot_scores_host, uint8_t* keep_host,
                                  int32_t* kept_idx_host, int32_t* kept_count_host, int32_t Mcap, shotkv_bf16* Kc_host,
                                  shotkv_bf16* Vc_host, void* arena, size_t arena_bytes, void* stream_) {
+    TraceRange trace_("shotkv_prefill_compress_host");
     int rc = set_device(ctx);
     if (rc) return rc;
     const char* why = "";
@@ -1227,12 +1244,14 @@ extern "C" {
 
 int shotkv_decode_step(shotkv_ctx* ctx, shotkv_decode_state* st, const shotkv_bf16* q, const shotkv_bf16* k_new,
                        const shotkv_bf16* v_new, const shotkv_bf16* Kc, const int32_t* kept_count, void* stream) {
+    TraceRange trace_("shotkv_decode_step");
     return decode_step_impl(ctx, st, q, k_new, v_new, Kc, nullptr, kept_count, nullptr, stream);
 }
 
 int shotkv_decode_step_attend(shotkv_ctx* ctx, shotkv_decode_state* st, const shotkv_bf16* q, const shotkv_bf16* k_new,
                               const shotkv_bf16* v_new, const shotkv_bf16* Kc, const shotkv_bf16* Vc,
                               const int32_t* kept_count, float* attn_out, void* stream) {
+    TraceRange trace_("shotkv_decode_step_attend");
     if (!attn_out) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "attn_out must not be NULL");
     return decode_step_impl(ctx, st, q, k_new, v_new, Kc, Vc, kept_count, attn_out, stream);
 }
@@ -1280,6 +1299,7 @@ int shotkv_set_wait_limit(shotkv_ctx* ctx, int64_t cycles) {
 }
 
 int shotkv_selftest_bounded_wait(shotkv_ctx* ctx, int64_t limit_cycles, int32_t* report, void* stream_) {
+    TraceRange trace_("shotkv_selftest_bounded_wait");
     int rc = set_device(ctx);
     if (rc) return rc;
     if (!report) return fail(ctx, SHOTKV_ERR_INVALID_ARG, "report must not be NULL");
