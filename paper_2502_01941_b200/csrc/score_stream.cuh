@@ -150,22 +150,27 @@ __global__ void __launch_bounds__(ScoreStreamCfg<D>::kThreads, 1)
             // 32 columns starting at key kc that hold the end of the keys, the causal window, or a piece end
             auto chunk_slow = [&](uint32_t (&r)[32], int kc) {
                 while (pend <= kc) flush();
-                if (kc + 32 <= plain_end && pend_n >= kc + 32) {
-                    // every column counts and at most one piece ends inside: the exponentials of the columns
-                    // before the end go to the current piece, the others start the next one
+                if (kc + 32 <= plain_end) {
+                    // every column counts; one or more pieces end inside.  Peel them off in order: the
+                    // columns before a piece's end go to its sum through a 0/1 mask, and the complementary
+                    // mask clears them from the chunk before the next piece is looked at.
                     tc::exp32_mixed<PE>(r, scale, neg);
-                    const float4* mk = mtab + min(pend - kc, 32) * 16;
-                    uint64_t h[2] = {0ull, 0ull};
+                    while (pend < kc + 32) {
+                        const float4* mk = mtab + (pend - kc) * 16;
 #pragma unroll
-                    for (int q = 0; q < 16; ++q) {
-                        const float4 m4 = mk[q];
-                        const uint64_t e2 = tc::pack2(SKV_F(r, 2 * q), SKV_F(r, 2 * q + 1));
-                        z[q & 1] = tc::ffma2(e2, tc::pack2(m4.x, m4.y), z[q & 1]);
-                        h[q & 1] = tc::ffma2(e2, tc::pack2(m4.z, m4.w), h[q & 1]);
+                        for (int q = 0; q < 16; ++q) {
+                            const float4 m4 = mk[q];
+                            const uint64_t e2 = tc::pack2(SKV_F(r, 2 * q), SKV_F(r, 2 * q + 1));
+                            z[q & 1] = tc::ffma2(e2, tc::pack2(m4.x, m4.y), z[q & 1]);
+                            float ea, eb;
+                            tc::unpack2(tc::ffma2(e2, tc::pack2(m4.z, m4.w), 0ull), ea, eb);
+                            r[2 * q] = __float_as_uint(ea);
+                            r[2 * q + 1] = __float_as_uint(eb);
+                        }
+                        flush();
                     }
-                    if (pend < kc + 32) flush();
-                    z[0] = tc::fadd2(z[0], h[0]);
-                    z[1] = tc::fadd2(z[1], h[1]);
+#pragma unroll
+                    for (int q = 0; q < 16; ++q) z[q & 1] = tc::fadd2(z[q & 1], tc::pack2(SKV_F(r, 2 * q), SKV_F(r, 2 * q + 1)));
                     return;
                 }
                 const int lim = min(hi, plim + 1) - kc;                  // columns of the chunk that count

@@ -399,6 +399,34 @@ def test_sentence_sized_units_full_path(ctx):
         assert int(gpu["kept_count"].max()) <= O.budget_tokens(cfg.r_p, cfg.N)
 
 
+def test_several_piece_ends_inside_one_chunk_of_256_row_units(ctx):
+    """Units of a handful of tokens next to long ones, on 256 window rows (the streaming kernel): runs
+    of very short units put two to five piece ends into one 32-column chunk of the scoring pass,
+    some exactly on chunk and tile boundaries, while the mean length keeps the call on its
+    single-pass route."""
+    N, W, S = 6000, 64, 40
+    rng = np.random.default_rng(17)
+    lens = []
+    while len(lens) < S:
+        lens += [int(x) for x in rng.integers(3, 12, size=4)] + [int(rng.integers(250, 420))]
+    lens = lens[:S]
+    # pin two ends onto a tile boundary and onto the chunk boundary after it
+    lens[4] = 384 - (32 + sum(lens[:4]))
+    lens[5] = 32
+    off = np.concatenate([[32], 32 + np.cumsum(lens)]).astype(np.int32)
+    assert off[5] == 384 and off[6] == 416
+    assert np.all(np.diff(off) > 0) and off[-1] <= N - W and N / S >= 40
+    ends_per_chunk = np.bincount(off[1:] // 32)
+    assert ends_per_chunk.max() >= 3, "the case needs several piece ends in one chunk"
+    cfg = wl.PrefillConfig("runs_of_tiny_units", B=2, L=1, H=32, Hkv=8, d=128, N=N, W=W, S=S, shot_dist="uniform", shot_lo=1,
+                           shot_hi=N, question_len=N - int(off[-1]), preamble_len=32, r_p=0.3, cfg_id=33)
+    offs = np.stack([off, off])
+    Q, K, V, _ = wl.prefill_batch(cfg, "cuda", offsets=offs)
+    for mode in (0, 1):
+        gpu = P.gpu_prefill(ctx, P.dims_of(cfg), Q, K, V, offs, cfg.r_p, mode, "fused")
+        assert P.check_all_units(gpu, Q, K, V, offs, cfg.r_p, mode) <= 2
+
+
 def test_fixed_size_chunks_as_units(ctx):
     """Chunk-level retention: the units are fixed-size chunks, off[i] = preamble + i*c."""
     c, N, W, q_len, pre = 16, 8192, 64, 200, 8
