@@ -1,23 +1,23 @@
-// Window attention scoring, the kernel the prefill path runs first: the same TMA producer, MMA
-// issuer, work items and per-(piece, window row) outputs (m, z) as score_tc.cuh, with an epilogue
-// arranged for throughput.
+// Window attention scoring for units of 128 window rows or fewer (one 128-row block of Q), the
+// kernel the prefill path runs first on them: the same TMA producer, MMA issuers, work items and
+// per-(piece, window row) outputs (m, z) as score_tc.cuh, with an epilogue arranged for
+// throughput.  (Units of more than 128 rows go to score_stream.cuh, which shares the exponential
+// helpers defined here.)
 //
-//   * Eight epilogue warps of up to 168 registers.  With 256 window rows a warp group owns a row
-//     block and every thread one whole row of a tile (four tensor-memory loads of 32 columns),
-//     so a piece's (m, z) is written by one thread with no exchange.  With 128 rows the two
-//     groups split a tile's columns in halves; when a piece is complete the second group hands
-//     its (m, z) to the first through a small ring of shared-memory slots guarded by mbarriers,
-//     so no warp waits for another at a piece end unless it is a whole ring ahead of it.  The
-//     code of the inner loop is kept small and free of branches (one copy of the chunk
-//     arithmetic, one of the boundary handling): the warps of three roles share the
-//     instruction cache.
-//   * No running maximum.  The reference exponent m of a (row, work item) is fixed from the
-//     item's first tile: that tile's row maximum lands on 2^-32, and every later logit of the
-//     item is exponentiated against the same m.  fp32 leaves about 2^+158 above that point and
-//     2^-94 below it; what underflows is below 2^-94 of a term the row's own softmax denominator
-//     contains, so it cannot matter to any score.  What overflows is caught: a partial sum that
-//     is not below 1e30 marks its item in `redo`, and a second launch (the exact kernel of
-//     score_tc.cuh with the same flags) recomputes marked items with a true running maximum.
+//   * Eight epilogue warps in two groups that split a tile's columns in halves; a thread is one
+//     window row and one half.  When a piece is complete the second group hands its (m, z) to the
+//     first through a small ring of shared-memory slots guarded by mbarriers, so no warp waits
+//     for another at a piece end unless it is a whole ring ahead of it.  The code of the inner
+//     loop is kept small and free of branches (one copy of the chunk arithmetic, one of the
+//     boundary handling): the warps of three roles share the instruction cache.
+//   * No running maximum.  The reference exponent m of a (row, column half, work item) is fixed
+//     from the item's first tile: that tile's row maximum lands on 2^-32, and every later logit
+//     of the item is exponentiated against the same m.  fp32 leaves about 2^+158 above that point
+//     and 2^-94 below it; what underflows is below 2^-94 of a term the row's own softmax
+//     denominator contains, so it cannot matter to any score.  What overflows is caught: a
+//     partial sum that is not below 1e30 marks its item in `redo`, and a second launch (the exact
+//     kernel of score_tc.cuh with the same flags) recomputes marked items with a true running
+//     maximum.
 //   * One ex2 per logit is the ceiling of the special-function unit (16 lanes per clock per SM),
 //     so PE of every 16 column pairs take their exponentials on the FMA pipe instead: round to nearest
 //     integer n by the magic-number addition, a cubic in the remainder f in [-1/2, 1/2]
@@ -29,19 +29,19 @@
 
 namespace shotkv {
 
-template <int D, int MB>
+template <int D>
 struct ScoreFastCfg {
     static constexpr int kSub = D / 64;
     static constexpr int kSubBytes = 128 * 128;
-    static constexpr int kQBytes = MB * kSub * kSubBytes;
+    static constexpr int kQBytes = kSub * kSubBytes;
     static constexpr int kStageBytes = kSub * kSubBytes;
-    static constexpr int kStages = D == 128 ? (MB == 2 ? 4 : 5) : 6;
+    static constexpr int kStages = D == 128 ? 5 : 6;
     static constexpr int kBarBytes = 2048;
     static constexpr int kRingDepth = 4;                       // hand-over slots between a row's column slices
-    static constexpr int kRings = 12;                          // (row block, warp quad, follower slice) triples, at most
+    static constexpr int kRings = 4;                           // one per warp quarter
     static constexpr int kCombBytes = kRings * kRingDepth * 32 * 2 * 4;   // [ring][slot][lane][m, z]
     static constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kBarBytes + kCombBytes + 1024;
-    static constexpr int kSlices = 2 / MB;                     // column slices of a tile
+    static constexpr int kSlices = 2;                          // column slices of a tile
     static constexpr int kEpiWarps = 8;
     static constexpr int kThreads = 128 + kEpiWarps * 32;      // producer, two MMA issuers, one idle warp; epilogue
 };
@@ -125,17 +125,17 @@ __device__ __forceinline__ void exp32_mixed(uint32_t (&r)[32], float scale, floa
 
 }  // namespace tc
 
-template <int D, int MB, int PE>
-__global__ void __launch_bounds__(ScoreFastCfg<D, MB>::kThreads, 1)
+template <int D, int PE>
+__global__ void __launch_bounds__(ScoreFastCfg<D>::kThreads, 1)
     score_fast_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const int q_box_rows,
                       const int k_box_rows, const ScoreTcParams p) {
-    using Cfg = ScoreFastCfg<D, MB>;
-    constexpr int TN = tc::kTileKeys;
+    using Cfg = ScoreFastCfg<D>;
+    constexpr int TN = tc::kTileKeys, MB = 1;
     constexpr int NSL = Cfg::kSlices, SLW = TN / NSL, NCH = SLW / 32, RD = Cfg::kRingDepth;
     extern __shared__ unsigned char smem_raw[];
     tc::stamp(p.clk, 0);
     tc::Pipe<Cfg> pp;
-    tc::pipe_setup(pp, smem_raw, Cfg::kEpiWarps / MB, Cfg::kRings * Cfg::kRingDepth * 2, 2);
+    tc::pipe_setup(pp, smem_raw, Cfg::kEpiWarps, Cfg::kRings * Cfg::kRingDepth * 2, 2);
     float* comb = tc::pipe_scratch(pp, smem_raw);     // [ring][slot][lane][m, z]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -151,9 +151,8 @@ __global__ void __launch_bounds__(ScoreFastCfg<D, MB>::kThreads, 1)
         // ------------------------------------------------------------------ epilogue
         // a warp may touch the 32 tensor-memory lanes given by its index modulo 4; any four
         // consecutive warps cover all 128 rows of a block
-        const int g = (warp - 4) >> 2, quad = warp & 3;
-        const int blk = MB == 2 ? g : 0;                   // 128-row block of Q
-        const int slice = MB == 2 ? 0 : g;                 // column slice of every tile
+        const int slice = (warp - 4) >> 2, quad = warp & 3;   // column slice of every tile, lane quarter
+        constexpr int blk = 0;                             // the one 128-row block of Q
         const int lrow = quad * 32 + lane;
         const int row = blk * 128 + lrow;
         const bool live = row < p.R;                       // padding rows: their Q was never loaded

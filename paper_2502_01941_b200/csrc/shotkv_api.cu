@@ -350,13 +350,13 @@ int launch_score_tc_t(shotkv_ctx* ctx, const CUtensorMap& tmQ, const CUtensorMap
 // Column pairs, of every 16, whose exponentials run on the FMA pipe instead of the special-function unit.
 constexpr int kPolyEvery = 5;
 
-template <int D, int MB>
+template <int D>
 int launch_score_fast_t(shotkv_ctx* ctx, const CUtensorMap& tmQ, const CUtensorMap& tmK, int qbox, int kbox,
                         const ScoreTcParams& sp, cudaStream_t stream) {
-    constexpr int smem = ScoreFastCfg<D, MB>::kSmemBytes;
+    constexpr int smem = ScoreFastCfg<D>::kSmemBytes;
     int grid = sp.total_items < ctx->sm_count ? sp.total_items : ctx->sm_count;
     if (grid < 1) grid = 1;
-    score_fast_kernel<D, MB, kPolyEvery><<<grid, ScoreFastCfg<D, MB>::kThreads, smem, stream>>>(tmQ, tmK, qbox, kbox, sp);
+    score_fast_kernel<D, kPolyEvery><<<grid, ScoreFastCfg<D>::kThreads, smem, stream>>>(tmQ, tmK, qbox, kbox, sp);
     LAUNCH_CHECK(ctx);
     return SHOTKV_OK;
 }
@@ -467,8 +467,8 @@ int launch_score_tc(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q,
         sp.redo_any = w.redo;
         sp.redo = w.redo + 1;
         CUDA_TRY(ctx, cudaMemsetAsync(w.redo, 0, ((size_t)sp.total_items + 1) * 4, stream));
-        if (d->d == 128) rc = big ? launch_score_stream_t<128>(ctx, tmQ, tmK, qbox, kbox, sp, stream) : launch_score_fast_t<128, 1>(ctx, tmQ, tmK, qbox, kbox, sp, stream);
-        else rc = big ? launch_score_stream_t<64>(ctx, tmQ, tmK, qbox, kbox, sp, stream) : launch_score_fast_t<64, 1>(ctx, tmQ, tmK, qbox, kbox, sp, stream);
+        if (d->d == 128) rc = big ? launch_score_stream_t<128>(ctx, tmQ, tmK, qbox, kbox, sp, stream) : launch_score_fast_t<128>(ctx, tmQ, tmK, qbox, kbox, sp, stream);
+        else rc = big ? launch_score_stream_t<64>(ctx, tmQ, tmK, qbox, kbox, sp, stream) : launch_score_fast_t<64>(ctx, tmQ, tmK, qbox, kbox, sp, stream);
         if (rc) return rc;
         sp.clk = nullptr;
     }
@@ -615,8 +615,9 @@ int run_compact(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* K, con
 template <int D, int MB>
 cudaError_t set_tc_attributes() {
     cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<D, MB>, cudaFuncAttributeMaxDynamicSharedMemorySize, ScoreTcCfg<D, MB>::kSmemBytes);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(score_fast_kernel<D, MB, kPolyEvery>, cudaFuncAttributeMaxDynamicSharedMemorySize, ScoreFastCfg<D, MB>::kSmemBytes);
+    // the first scoring launch: one 128-row block of Q -> score_fast_kernel, two -> score_stream_kernel
+    if (e == cudaSuccess && MB == 1)
+        e = cudaFuncSetAttribute(score_fast_kernel<D, kPolyEvery>, cudaFuncAttributeMaxDynamicSharedMemorySize, ScoreFastCfg<D>::kSmemBytes);
     if (e == cudaSuccess && MB == 2)
         e = cudaFuncSetAttribute(score_stream_kernel<D, kPolyEvery>, cudaFuncAttributeMaxDynamicSharedMemorySize, ScoreStreamCfg<D>::kSmemBytes);
     if (e == cudaSuccess)
