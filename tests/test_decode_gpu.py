@@ -242,3 +242,32 @@ def test_decode_config4_all_1024_steps_two_units(ctx, attend):
     ties = lockstep(ctx, cfg, 3276, [(1, 4), (6, 29)], attend=attend)
     assert lockstep.largest_region >= 279
     assert ties <= 6
+
+
+def _random_decode_cases(n, seed):
+    rng = np.random.default_rng(seed)
+    cases = []
+    for i in range(n):
+        Hkv = int(rng.choice([1, 2, 3]))
+        G = int(rng.choice([1, 2, 3, 4, 6, 8]))
+        cases.append((wl.DecodeConfig(f"rdec{i}", B=int(rng.choice([1, 2])), L=int(rng.choice([1, 2])), H=G * Hkv, Hkv=Hkv,
+                                      d=int(rng.choice([64, 128])), steps=int(rng.integers(20, 70)),
+                                      r_d=float(rng.choice([0.2, 0.5, 0.75, 1.0])), recompress_every=int(rng.choice([1, 3, 8, 16])),
+                                      cfg_id=800 + i),
+                      int(rng.choice([0, 1, 15, 16, 17, 130, 500])), int(rng.choice([0, 0, 2]))))
+    return cases
+
+
+RANDOM_DECODE = _random_decode_cases(8, seed=20250202)
+
+
+@pytest.mark.parametrize("attend", [False, True], ids=["plain", "attend"])
+@pytest.mark.parametrize("cfg,M,protect", RANDOM_DECODE, ids=[f"{c.name}_g{c.H // c.Hkv}_d{c.d}_m{m}" for c, m, _ in RANDOM_DECODE])
+def test_random_decode_shapes(ctx, cfg, M, protect, attend):
+    """Seeded random shapes: group sizes that are not powers of two, prefill regions of 0, 1, one
+    block, one block and a row, and many rows; every step checked against the oracle."""
+    counts = None
+    if M == 0:
+        counts, M = np.zeros((cfg.B, cfg.L), np.int32), 4
+    units = [(b, l) for b in range(cfg.B) for l in range(cfg.L)]
+    assert lockstep(ctx, cfg, M, units, counts, attend=attend, protect_recent=protect) <= 3

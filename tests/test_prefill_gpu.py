@@ -535,3 +535,41 @@ def test_host_buffer_entry_point_pipelined(ctx):
         skv.shotkv_set_pipeline_groups(ctx, 0)
     hout["token_importance"] = None
     P.check_all_units(hout, Q, K, V, off, cfg.r_p)
+
+
+def _random_prefill_cases(n, seed):
+    """Seeded random shapes across the supported range: both head dimensions, 1 to 256 window rows,
+    N not a multiple of anything, one to many units (short ones too), preamble or none, both select modes."""
+    rng = np.random.default_rng(seed)
+    cases = []
+    while len(cases) < n:
+        d = int(rng.choice([64, 128]))
+        Hkv = int(rng.choice([1, 2, 4]))
+        G = int(rng.choice([1, 2, 4, 8]))
+        W = int(rng.choice([w for w in (1, 3, 8, 16, 32, 64, 100, 128) if G * w <= 256]))
+        N = int(rng.integers(max(W + 40, 150), 2600))
+        S = int(rng.integers(1, 14))
+        pre = int(rng.choice([0, 0, 5, 33]))
+        q_len = int(rng.integers(W, W + 60))
+        room = N - q_len - pre
+        if room < 2 * S:
+            continue
+        lo = max(1, room // (3 * S))
+        hi = max(lo, min(room - lo * (S - 1), 3 * room // S))
+        cases.append(wl.PrefillConfig(f"rand{len(cases)}_d{d}_g{G}_w{W}_n{N}_s{S}", B=int(rng.choice([1, 2])), L=int(rng.choice([1, 2])),
+                                      H=G * Hkv, Hkv=Hkv, d=d, N=N, W=W, S=S, shot_dist="uniform", shot_lo=lo, shot_hi=hi,
+                                      question_len=q_len, preamble_len=pre, r_p=float(rng.choice([0.15, 0.35, 0.6, 0.9])),
+                                      cfg_id=700 + len(cases)))
+    return cases
+
+
+RANDOM_CASES = _random_prefill_cases(14, seed=20250201)
+
+
+@pytest.mark.parametrize("cfg", RANDOM_CASES, ids=[c.name for c in RANDOM_CASES])
+def test_random_shapes_all_paths(ctx, cfg):
+    """Every path on shapes nobody picked by hand; the select mode alternates with the case."""
+    mode = cfg.cfg_id & 1
+    for path in PATHS:
+        ties, _ = run_cfg(ctx, cfg, path, select_mode=mode)
+        assert ties <= 2
