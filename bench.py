@@ -184,10 +184,11 @@ def run_ours(args):
     if args.units == "sentences":       # same tensors' shapes, units of 10-40 tokens
         cfg = cfg.replace(S=(cfg.N - cfg.question_len) // 25, shot_dist="uniform", shot_lo=10, shot_hi=40,
                           name=cfg.name + "[sentence units]")
-    elif args.units == "chunks":        # fixed chunks of 16 tokens; the remainder joins the question
-        S = (cfg.N - cfg.question_len) // 16
-        cfg = cfg.replace(S=S, shot_dist="uniform", shot_lo=16, shot_hi=16, question_len=cfg.N - 16 * S,
-                          name=cfg.name + "[16-token chunks]")
+    elif args.units == "chunks":        # fixed chunks of --chunk-tokens tokens (16); the remainder joins the question
+        c = args.chunk_tokens
+        S = (cfg.N - cfg.question_len) // c
+        cfg = cfg.replace(S=S, shot_dist="uniform", shot_lo=c, shot_hi=c, question_len=cfg.N - c * S,
+                          name=cfg.name + f"[{c}-token chunks]")
     dims = skv.make_dims(cfg.B, cfg.L, cfg.H, cfg.Hkv, cfg.d, cfg.N, cfg.W, cfg.S)
     pol = skv.make_policy(r_p=cfg.r_p)
     Q, K, V, off = wl.prefill_batch(cfg, dev)
@@ -623,6 +624,7 @@ def main():
     ap.add_argument("--units", default="shots", choices=["shots", "sentences", "chunks"],
                     help="semantic units of the timed workload: the config's few-shot examples (default), sentence-sized "
                          "units of 10-40 tokens (the document-QA adaptation), or fixed chunks of 16 tokens")
+    ap.add_argument("--chunk-tokens", type=int, default=16, help="chunk length for --units chunks")
     ap.add_argument("--scoring", default="fast", choices=sorted(SCORING_MODES),
                     help="scoring kernel: the default pair (fast kernel + exact repair) or the exact kernel alone")
     ap.add_argument("--groups", type=int, default=0, choices=[0, 1, 2, 3, 4],

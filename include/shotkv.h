@@ -173,9 +173,12 @@ SHOTKV_API int shotkv_compact_kv(shotkv_ctx* ctx, const shotkv_dims* dims,
  * SHOTKV_FLAG_TOKEN_IMPORTANCE the shot scores are formed directly from per-shot partial sums
  * (K is streamed once and per-token importance is never materialised; token_importance is
  * ignored and may be NULL); with it the call equals the three calls above in sequence.
- * When the units are short (fewer than 40 tokens on average, e.g. sentence-sized units or fixed
- * chunks) the call also goes through per-token importances, kept in the workspace: the cost of
- * that route does not grow with S.  Arguments as in those calls.
+ * When the units are very short (fewer than 16 tokens on average with more than 128 window rows
+ * G*W, fewer than 40 otherwise) the call also goes through per-token importances, kept in the
+ * workspace: the cost of that route does not grow with S.  Longer units -- with 256 window rows
+ * that includes sentence-sized units and 16-token chunks -- stay on the single-pass form, whose
+ * workspace grows with S (two floats per unit, window row and KV head).  Arguments as in those
+ * calls.
  *   Units (b, l) are independent (Algorithm 1 compresses layer by layer), so the single-pass form
  *   can cut them into up to four groups -- whole prompts, or runs of layers when B = 1 -- and
  *   reduce, select and compact one group on a stream the context owns while `stream` works on the

@@ -175,6 +175,7 @@ __global__ void __launch_bounds__(ScoreFastCfg<D>::kThreads, 1)
             int pend = pi < pi_last ? pcs[pi].y : 0x7fffffff;
             int pend_n = pi + 1 < pi_last ? pcs[pi + 1].y : 0x7fffffff;
             float m_ref = SHOTKV_NEG_INF, neg = 0.f;       // reference exponent of this (row, slice, item); neg = -m_ref
+            float item_mm = SHOTKV_NEG_INF, item_zz = 0.f; // leader: the row's statistics over the item's pieces so far
             uint64_t z[2] = {0ull, 0ull};                  // four running sums of the current piece, as two packed pairs
             const int plain_end = min(hi, p.N - p.W + 1);  // keys below this count for every window row
 
@@ -230,9 +231,16 @@ __global__ void __launch_bounds__(ScoreFastCfg<D>::kThreads, 1)
                     if (NSL > 1) zz *= ex2f(m_ref - mu);
 #pragma unroll
                     for (int s = 1; s < NSL; ++s) zz += zs[s - 1] * ex2f(ms[s - 1] - mu);
+                    // the merged reference is the larger of the slices' references, both fixed on the item's
+                    // first tile: the same for every piece of the item, so only z goes out per piece
                     const size_t o = ((size_t)u * p.P + pi) * p.Rpad + row;
-                    p.part_m[o] = live ? mm : 0.f;
                     p.part_z[o] = live ? zz : 0.f;
+                    {
+                        const float mn = fmaxf(item_mm, mm);
+                        const float mq = mn == SHOTKV_NEG_INF ? 0.f : mn;
+                        item_zz = item_zz * ex2f(item_mm - mq) + zz * ex2f(mm - mq);
+                        item_mm = mn;
+                    }
                 }
                 z[0] = z[1] = 0ull;
                 ++nflush;
@@ -324,6 +332,10 @@ __global__ void __launch_bounds__(ScoreFastCfg<D>::kThreads, 1)
             }
             if (!ok) break;
             while (pi < pi_last) flush();
+            if (slice == 0) {
+                p.item_m[(size_t)it * p.Rpad + row] = live ? item_mm : 0.f;
+                p.item_z[(size_t)it * p.Rpad + row] = live ? item_zz : 0.f;
+            }
         }
     }
 

@@ -5,7 +5,7 @@
 // waits for tensor memory.
 //
 // Eight epilogue warps, one per (row block, tensor-memory lane quarter); a thread is one whole
-// window row, so a piece's (m, z) is written by one thread with no exchange.  The accumulator
+// window row, so a piece's z (and the item's reference m) is written by one thread with no exchange.  The accumulator
 // columns of the next 32-column chunk -- of the next tile too, once its barrier is seen complete
 // -- are requested into a second set of registers before the arithmetic of the current chunk
 // starts, so the load's latency runs beside the exponentials.  Where a piece ends inside a chunk
@@ -13,10 +13,13 @@
 // from a shared-memory table (one packed multiply-add per column pair and piece), which costs
 // half the instructions of a predicated addition per column.
 //
-// What bounds this kernel on a power-capped B200 is energy, not a pipe: see the measurements in
-// the repository's design notes.  The share of the exponentials on the FMA pipe (PE of every 16
-// column pairs) is therefore small here: the polynomial costs 5.5 issue slots per logit against
-// 2 for the special-function path.
+// What bounds this kernel on a B200 held at a 1 kW power cap is energy per tile, not a pipe: its
+// epilogue takes the same cycles per tile with or without the MMAs running beside it, but the GPU
+// settles near 1.5 GHz with them and at its full 1.96 GHz without.  The polynomial costs 5.5 issue
+// slots per logit against 2 for the special-function path, so a larger share on the FMA pipe
+// (PE of every 16 column pairs) saves cycles and spends energy; measured at the cap, shares from 2
+// to 5 of 16 come out within the noise of the power controller, and below the cap the larger
+// share is faster.
 #pragma once
 #include "score_fast.cuh"
 
@@ -123,8 +126,8 @@ __global__ void __launch_bounds__(ScoreStreamCfg<D>::kThreads, 1)
             float m_ref = SHOTKV_NEG_INF, neg = 0.f;       // reference exponent of this (row, item); neg = -m_ref
             uint64_t z[2] = {0ull, 0ull};                  // four running sums of the current piece, as two packed pairs
             const int plain_end = min(hi, p.N - p.W + 1);  // keys below this count for every window row
-            float* out_m = p.part_m + ((size_t)u * p.P + pi) * p.Rpad + row;
             float* out_z = p.part_z + ((size_t)u * p.P + pi) * p.Rpad + row;
+            float zsum = 0.f;                              // sum of the item's pieces so far (they share m_ref)
 
             // piece `pi` is complete: write its partials and move on to the next piece
             auto flush = [&]() {
@@ -137,10 +140,9 @@ __global__ void __launch_bounds__(ScoreStreamCfg<D>::kThreads, 1)
                     p.redo[it] = 1;
                     *p.redo_any = 1;
                 }
-                *out_m = live ? m_ref : 0.f;
                 *out_z = live ? zz : 0.f;
-                out_m += p.Rpad;
                 out_z += p.Rpad;
+                zsum += zz;
                 z[0] = z[1] = 0ull;
                 ++pi;
                 pend = pend_n;
@@ -264,6 +266,9 @@ __global__ void __launch_bounds__(ScoreStreamCfg<D>::kThreads, 1)
             }
             if (!ok) break;
             while (pi < pi_last) flush();
+            // the row's statistics over the whole item: its reference and the sum of its pieces
+            p.item_m[(size_t)it * p.Rpad + row] = live ? m_ref : 0.f;
+            p.item_z[(size_t)it * p.Rpad + row] = live ? zsum : 0.f;
             tiles_before += nt;
         }
         // an abort may leave a requested chunk unread: nothing of tensor memory is in flight past here

@@ -41,8 +41,10 @@ struct ScoreTcParams {
     int L, Hkv, N, W, R, Rpad;
     int total_items;          // U * nchunk
     float scale_log2;     // log2(e)/sqrt(d)
-    float* part_m;        // [U][P][Rpad]
+    float* part_m;        // [U][P][Rpad]  per-piece reference: written by the exact kernel only
     float* part_z;        // [U][P][Rpad]
+    float* item_m;        // [U * nchunk][Rpad]  the one reference of an item's pieces, and the sum of their z:
+    float* item_z;        //                     written by the kernels that fix a reference per item
     int* err;             // error word (host-visible); set to 1 when a bounded wait gave up
     long long wait_cycles;    // limit of every bounded wait, in SM clock cycles
     long long* clk;           // optional (host-visible): SM cycle counter and nanosecond timer of CTA 0 at kernel start and end

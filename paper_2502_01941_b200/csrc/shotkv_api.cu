@@ -175,12 +175,18 @@ int check_offsets(const shotkv_dims* d, const shotkv_policy* p, const int32_t* o
 }
 
 int rpad_of(const shotkv_dims* d) { return (d->H / d->Hkv) * d->W <= 128 ? 128 : 256; }
-// Units shorter than this many tokens on average put a piece end in most 32-column chunks of the
-// scoring pass and make its per-piece partials a sizeable fraction of K; the fused call then goes
-// through per-token importances instead (two passes over K, cost independent of S), which
-// measures faster from about this point on.
-constexpr int kTokenRouteBelowMeanLen = 40;
-bool token_route(const shotkv_dims* d) { return d->S > 0 && (long long)d->N < (long long)kTokenRouteBelowMeanLen * d->S; }
+// Units shorter than this many tokens on average put several piece ends into every 32-column chunk
+// of the scoring pass; the fused call then goes through per-token importances instead (two passes
+// over K, cost independent of S).  Measured on 4 x 32 layers x 32,768 tokens: sentence-sized units
+// (25 tokens on average) 5.7 ms single-pass against 6.8 ms two-pass, 16-token chunks 6.0 against
+// 6.9, 12-token chunks 8.3 against 7.1, 8-token chunks 10.5 against 7.5.
+// The kernel for 128 window rows or fewer still splits its chunks by predicated additions, which
+// cost more per piece end; there the two-pass route wins from 40 tokens down, as measured before.
+constexpr int kTokenRouteBelowMeanLen = 16, kTokenRouteBelowMeanLenFewRows = 40;
+bool token_route(const shotkv_dims* d) {
+    const int below = rpad_of(d) > 128 ? kTokenRouteBelowMeanLen : kTokenRouteBelowMeanLenFewRows;
+    return d->S > 0 && (long long)d->N < (long long)below * d->S;
+}
 // Pieces per prompt the workspace is sized for: shot boundaries plus chunk ends, or chunk ends alone
 // when the shot-aware scoring pass is never run for these dims.
 int pmax_of(const shotkv_dims* d) { return (token_route(d) ? 0 : d->S) + 2 + kMaxChunks + 1; }
@@ -192,6 +198,8 @@ struct PrefillWs {
     int* chunk_first;  // [B][kMaxChunks + 1]
     float* part_m;     // [U][Pmax][Rpad]
     float* part_z;
+    float* item_m;     // [U * kMaxChunks][Rpad] per (work item, row): the reference its pieces share and the sum of their z
+    float* item_z;
     float* row_m;      // [U][Rpad]
     float* row_invz;
     float* unit_shot;  // [U][S]
@@ -211,6 +219,8 @@ PrefillWs carve(const shotkv_dims* d, void* base) {
     w.chunk_first = (int*)take((size_t)d->B * (kMaxChunks + 1) * 4);
     w.part_m = (float*)take(U * P * R * 4);
     w.part_z = (float*)take(U * P * R * 4);
+    w.item_m = (float*)take(U * kMaxChunks * R * 4);
+    w.item_z = (float*)take(U * kMaxChunks * R * 4);
     w.row_m = (float*)take(U * R * 4);
     w.row_invz = (float*)take(U * R * 4);
     w.unit_shot = (float*)take(U * (size_t)(d->S > 0 ? d->S : 1) * 4);
@@ -418,6 +428,7 @@ int tc_setup(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const 
     sp.total_items = (int)(U * plan.nchunk);
     sp.scale_log2 = kLog2e / sqrtf((float)d->d);
     sp.part_m = w.part_m; sp.part_z = w.part_z;
+    sp.item_m = w.item_m; sp.item_z = w.item_z;
     sp.err = ctx->err_dev;
     sp.wait_cycles = ctx->wait_cycles;
     sp.repaired = ctx->err_dev + 1;
@@ -501,6 +512,20 @@ int prepare_pieces(shotkv_ctx* ctx, const shotkv_dims* d, const int32_t* off_hos
     return SHOTKV_OK;
 }
 
+// What the scoring pass just left in `w`, as the reductions read it.
+PartialView partial_view(const shotkv_ctx* ctx, const shotkv_dims* d, const PrefillWs& w, int P, const ChunkPlan& plan) {
+    PartialView v{};
+    v.part_m = w.part_m; v.part_z = w.part_z; v.item_m = w.item_m; v.item_z = w.item_z;
+    v.all_exact = ctx->scoring_mode == SHOTKV_SCORING_EXACT ? 1 : 0;
+    v.redo = v.all_exact ? nullptr : w.redo + 1;
+    v.chunk_first = w.chunk_first;
+    v.cf_stride = kMaxChunks + 1;
+    v.nchunk = plan.nchunk;
+    v.P = P;
+    v.Rpad = rpad_of(d);
+    return v;
+}
+
 // STATS pass over `pieces` followed by the per-row reduction; leaves part_m/part_z (and for the
 // token path row_m/row_invz) in the workspace.
 int run_stats(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const shotkv_bf16* K, const PrefillWs& w,
@@ -515,8 +540,7 @@ int run_stats(shotkv_ctx* ctx, const shotkv_dims* d, const shotkv_bf16* Q, const
     if (rc) return rc;
     prof_mark(ctx, stream);
     if (need_rows) {
-        row_stats_kernel<<<U, 256, 0, stream>>>(w.part_m, w.part_z, w.piece_seg, d->L * d->Hkv, d->S + 1, P, (d->H / d->Hkv) * d->W, rpad_of(d),
-                                                w.row_m, w.row_invz);
+        row_stats_kernel<<<U, 256, 0, stream>>>(partial_view(ctx, d, w, P, plan), d->L * d->Hkv, (d->H / d->Hkv) * d->W, w.row_m, w.row_invz);
         LAUNCH_CHECK(ctx);
     }
     *P_out = P;
@@ -578,6 +602,8 @@ PrefillWs group_ws(const PrefillWs& w, const shotkv_dims* d, const GroupView& v,
     x.chunk_first = w.chunk_first + v.b0 * (kMaxChunks + 1);
     x.part_m = w.part_m + v.u0 * P * R;
     x.part_z = w.part_z + v.u0 * P * R;
+    x.item_m = w.item_m + v.u0 * kMaxChunks * R;
+    x.item_z = w.item_z + v.u0 * kMaxChunks * R;
     x.row_m = w.row_m + v.u0 * R;
     x.row_invz = w.row_invz + v.u0 * R;
     x.unit_shot = w.unit_shot + v.u0 * (size_t)(d->S > 0 ? d->S : 1);
@@ -937,7 +963,7 @@ int prefill_compress_impl(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv
     if ((rc = upload_small(ctx, w.off, offsets_host, (size_t)dims->B * (S + 1) * 4, stream))) return rc;
     int P = 0;
     if ((rc = prepare_pieces(ctx, dims, offsets_host, plan, w, &P, stream))) return rc;
-    const size_t msm = (size_t)P * (Rpad / 32 + 1) * 4;
+    const size_t msm = ((size_t)P + 2 * Rpad) * 4;     // shot_mass_kernel: row statistics and one mass per piece
     if (S > 0) {
         if (msm > kBigSmem) return fail(ctx, SHOTKV_ERR_UNSUPPORTED_SHAPE, "too many shots for the single-pass path (S = %d)", S);
     }
@@ -972,10 +998,11 @@ int prefill_compress_impl(shotkv_ctx* ctx, const shotkv_dims* dims, const shotkv
         }
         prof_gmark(ctx, g, 2, tail);
         if (S > 0) {
+            const PartialView pv = partial_view(ctx, dg, wg, P, plan);
             if (Rpad == 128)
-                shot_mass_kernel<128><<<Ug, 128, msm, tail>>>(wg.part_m, wg.part_z, wg.piece_seg, P, R, Rpad, dg->L, dg->Hkv, S, wg.unit_shot);
+                shot_mass_kernel<128><<<Ug, 128, msm, tail>>>(pv, wg.piece_seg, R, dg->L, dg->Hkv, S, wg.unit_shot);
             else
-                shot_mass_kernel<256><<<Ug, 256, msm, tail>>>(wg.part_m, wg.part_z, wg.piece_seg, P, R, Rpad, dg->L, dg->Hkv, S, wg.unit_shot);
+                shot_mass_kernel<256><<<Ug, 256, msm, tail>>>(pv, wg.piece_seg, R, dg->L, dg->Hkv, S, wg.unit_shot);
             ctx->launches += 1;
             if (cudaGetLastError() != cudaSuccess) return bail(fail(ctx, SHOTKV_ERR_CUDA, "per-shot reduction failed to launch"));
             shot_score_from_mass_kernel<<<dg->B * dg->L, 128, 0, tail>>>(wg.unit_shot, wg.off, dg->L, dg->Hkv, S, scores_g);

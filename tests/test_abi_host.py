@@ -140,17 +140,24 @@ def test_scoring_work_partition_covers_every_key_once(cid):
 
 
 def test_short_units_size_the_workspace_for_the_per_token_route():
-    """Below a mean unit length of 40 tokens the fused call goes through per-token importances, and
-    the workspace holds those (U*N floats) instead of softmax partials for S + 67 pieces."""
+    """Below a mean unit length of 16 tokens (256 window rows; 40 tokens at 128 rows or fewer) the fused
+    call goes through per-token importances, and the workspace holds those (U*N floats) instead of
+    softmax partials for S + 67 pieces."""
     long_units = skv.make_dims(1, 2, 32, 8, 128, 32768, 64, 96)
-    short_units = skv.make_dims(1, 2, 32, 8, 128, 32768, 64, 1290)
-    edge_a = skv.make_dims(1, 2, 32, 8, 128, 32768, 64, 819)      # 32768 / 819 = 40.01: still the shot-aware route
-    edge_b = skv.make_dims(1, 2, 32, 8, 128, 32768, 64, 820)      # 39.96: per-token route
-    ws = {k: skv.shotkv_workspace_bytes(v) for k, v in dict(l=long_units, s=short_units, a=edge_a, b=edge_b).items()}
+    sentences = skv.make_dims(1, 2, 32, 8, 128, 32768, 64, 1290)      # 25 tokens on average: single-pass
+    tiny_units = skv.make_dims(1, 2, 32, 8, 128, 32768, 64, 4000)     # 8 tokens: per-token route
+    edge_a = skv.make_dims(1, 2, 32, 8, 128, 32768, 64, 2048)         # 32768 / 2048 = 16: still the shot-aware route
+    edge_b = skv.make_dims(1, 2, 32, 8, 128, 32768, 64, 2049)         # 15.99: per-token route
+    ws = {k: skv.shotkv_workspace_bytes(v) for k, v in dict(l=long_units, s=sentences, t=tiny_units, a=edge_a, b=edge_b).items()}
     U, N, R = 2 * 8, 32768, 256
-    assert ws["s"] < ws["a"] and ws["b"] < ws["a"]
-    assert ws["b"] >= U * N * 4 and ws["b"] < U * N * 4 + U * 80 * R * 8 + (1 << 20)
-    assert ws["a"] >= U * (819 + 2) * R * 8
+    assert ws["l"] < ws["s"] < ws["a"] and ws["t"] < ws["a"] and ws["b"] < ws["a"]
+    # per-token importances, softmax partials for at most 67 pieces, row statistics for at most 64 work items per unit
+    assert ws["b"] >= U * N * 4 and ws["b"] < U * N * 4 + U * (80 + 64) * R * 8 + (1 << 20)
+    assert ws["a"] >= U * (2048 + 2) * R * 8
+    assert ws["s"] >= U * (1290 + 2) * R * 8
+    few_rows_a = skv.make_dims(1, 2, 32, 8, 128, 32768, 32, 819)      # 128 window rows, 40.01 tokens: shot-aware route
+    few_rows_b = skv.make_dims(1, 2, 32, 8, 128, 32768, 32, 820)      # 39.96: per-token route
+    assert skv.shotkv_workspace_bytes(few_rows_b) < skv.shotkv_workspace_bytes(few_rows_a)
 
 
 def test_per_head_dims_reads_heads_as_layers():

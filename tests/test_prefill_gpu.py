@@ -60,6 +60,9 @@ SHRUNK = [
     # pieces longer than the scoring kernel's longest key range (one shot of > 512 tokens)
     wl.PrefillConfig("long_shots", B=1, L=1, H=8, Hkv=2, d=128, N=4000, W=16, S=3, shot_dist="uniform", shot_lo=1000,
                      shot_hi=1400, question_len=400, preamble_len=5, r_p=0.45, cfg_id=13),
+    # units of 5-20 tokens on 256 window rows: short enough for the per-token route even there
+    wl.PrefillConfig("tiny_units_256_rows", B=1, L=1, H=16, Hkv=4, d=128, N=2048, W=64, S=150, shot_dist="uniform", shot_lo=5,
+                     shot_hi=20, question_len=173, r_p=0.3, cfg_id=16),
     # sentence-sized units: many short segments, several per tile
     wl.PrefillConfig("short_units", B=1, L=1, H=8, Hkv=4, d=128, N=2048, W=8, S=60, shot_dist="uniform", shot_lo=10,
                      shot_hi=50, question_len=64, r_p=0.3, cfg_id=14),
@@ -328,12 +331,15 @@ def test_exact_scoring_mode(ctx, cfg):
     assert ties <= 2
 
 
+@pytest.mark.parametrize("H,W", [(16, 16), (32, 64)], ids=["32_rows", "256_rows"])
 @pytest.mark.parametrize("col", [3, 6])
-def test_fast_scoring_out_of_range_items_are_recomputed(ctx, col):
+def test_fast_scoring_out_of_range_items_are_recomputed(ctx, col, H, W):
     """A key whose logit lies thousands of nats above its work item's first tile leaves the fp32
-    range the fast kernel works in (on the special-function path for col 6, on the FMA path for
-    col 3); the item must be recomputed by the exact kernel and the result must still match."""
-    cfg = wl.PrefillConfig("outlier", B=1, L=8, H=16, Hkv=8, d=64, N=2048, W=16, S=6, shot_dist="uniform", shot_lo=200,
+    range the first scoring kernel works in (the fast kernel at 32 window rows, the streaming kernel
+    at 256; one column on the special-function path, the other on the FMA path); the item must be
+    recomputed by the exact kernel, the reductions must take that item's statistics from the
+    exact kernel's per-piece references, and the result must still match."""
+    cfg = wl.PrefillConfig("outlier", B=1, L=8, H=H, Hkv=8, d=64, N=2048, W=W, S=6, shot_dist="uniform", shot_lo=200,
                            shot_hi=400, question_len=100, r_p=0.5, cfg_id=21)
     Q, K, V, off = wl.prefill_batch(cfg, "cuda")
     dims = P.dims_of(cfg)
