@@ -33,7 +33,7 @@ struct ScoreStreamCfg {
     static constexpr int kStageBytes = kSub * kSubBytes;
     static constexpr int kStages = D == 128 ? 4 : 6;
     static constexpr int kBarBytes = 1024;
-    static constexpr int kCombBytes = 33 * 16 * 16;            // split masks: [columns of the first piece][column pair] float4
+    static constexpr int kCombBytes = tc::kSplitMaskBytes;     // split masks: [columns of the piece that ends][column pair] float4
     static constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kBarBytes + kCombBytes + 1024;
     static constexpr int kEpiWarps = 8;
     static constexpr int kThreads = 128 + kEpiWarps * 32;      // producer, two MMA issuers, one idle warp; epilogue
@@ -80,13 +80,8 @@ __global__ void __launch_bounds__(ScoreStreamCfg<D>::kThreads, 1)
     tc::stamp(p.clk, 0);
     tc::Pipe<Cfg> pp;
     tc::pipe_setup(pp, smem_raw, 4, 0, 2);
-    // split masks: entry (nb, j) = {col 2j < nb, col 2j+1 < nb, col 2j >= nb, col 2j+1 >= nb} as 1.0 / 0.0
-    float4* mtab = reinterpret_cast<float4*>(tc::pipe_scratch(pp, smem_raw));
-    for (int i = threadIdx.x; i < 33 * 16; i += blockDim.x) {
-        const int nb = i >> 4, j = i & 15;
-        const float a = 2 * j < nb ? 1.f : 0.f, b = 2 * j + 1 < nb ? 1.f : 0.f;
-        mtab[i] = make_float4(a, b, 1.f - a, 1.f - b);
-    }
+    float4* mtab = reinterpret_cast<float4*>(tc::pipe_scratch(pp, smem_raw));   // split masks
+    tc::build_split_masks(mtab);
     __syncthreads();
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -152,27 +147,8 @@ __global__ void __launch_bounds__(ScoreStreamCfg<D>::kThreads, 1)
             // 32 columns starting at key kc that hold the end of the keys, the causal window, or a piece end
             auto chunk_slow = [&](uint32_t (&r)[32], int kc) {
                 while (pend <= kc) flush();
-                if (kc + 32 <= plain_end) {
-                    // every column counts; one or more pieces end inside.  Peel them off in order: the
-                    // columns before a piece's end go to its sum through a 0/1 mask, and the complementary
-                    // mask clears them from the chunk before the next piece is looked at.
-                    tc::exp32_mixed<PE>(r, scale, neg);
-                    while (pend < kc + 32) {
-                        const float4* mk = mtab + (pend - kc) * 16;
-#pragma unroll
-                        for (int q = 0; q < 16; ++q) {
-                            const float4 m4 = mk[q];
-                            const uint64_t e2 = tc::pack2(SKV_F(r, 2 * q), SKV_F(r, 2 * q + 1));
-                            z[q & 1] = tc::ffma2(e2, tc::pack2(m4.x, m4.y), z[q & 1]);
-                            float ea, eb;
-                            tc::unpack2(tc::ffma2(e2, tc::pack2(m4.z, m4.w), 0ull), ea, eb);
-                            r[2 * q] = __float_as_uint(ea);
-                            r[2 * q + 1] = __float_as_uint(eb);
-                        }
-                        flush();
-                    }
-#pragma unroll
-                    for (int q = 0; q < 16; ++q) z[q & 1] = tc::fadd2(z[q & 1], tc::pack2(SKV_F(r, 2 * q), SKV_F(r, 2 * q + 1)));
+                if (kc + 32 <= plain_end) {                              // every column counts; pieces end inside
+                    tc::peel_chunk<PE>(r, scale, neg, mtab, kc, pend, z, flush);
                     return;
                 }
                 const int lim = min(hi, plim + 1) - kc;                  // columns of the chunk that count

@@ -180,8 +180,9 @@ int rpad_of(const shotkv_dims* d) { return (d->H / d->Hkv) * d->W <= 128 ? 128 :
 // over K, cost independent of S).  Measured on 4 x 32 layers x 32,768 tokens: sentence-sized units
 // (25 tokens on average) 5.7 ms single-pass against 6.8 ms two-pass, 16-token chunks 6.0 against
 // 6.9, 12-token chunks 8.3 against 7.1, 8-token chunks 10.5 against 7.5.
-// The kernel for 128 window rows or fewer still splits its chunks by predicated additions, which
-// cost more per piece end; there the two-pass route wins from 40 tokens down, as measured before.
+// With 128 window rows or fewer a pass over K costs half the exponentials and the work of splitting
+// chunks at piece ends weighs twice as much beside it: there the two-pass route wins from about 40
+// tokens down (1 x 32 layers x 16,384 tokens, sentence-sized units: 0.71 ms against 0.95 ms single-pass).
 constexpr int kTokenRouteBelowMeanLen = 16, kTokenRouteBelowMeanLenFewRows = 40;
 bool token_route(const shotkv_dims* d) {
     const int below = rpad_of(d) > 128 ? kTokenRouteBelowMeanLen : kTokenRouteBelowMeanLenFewRows;
