@@ -153,6 +153,29 @@ def rank_config(cfg: wl.PrefillConfig, rank: int) -> wl.PrefillConfig:
     return cfg if rank == 0 else cfg.replace(cfg_id=cfg.cfg_id + 1000 * rank)
 
 
+def units_variant(cfg, kind: str, chunk_tokens: int = 16):
+    """The workload with other semantic units: "sentences" = units of 10-40 tokens, "chunks" = fixed
+    chunks of `chunk_tokens` tokens (the remainder joins the question), "shots" = as configured."""
+    if kind == "sentences":
+        return cfg.replace(S=(cfg.N - cfg.question_len) // 25, shot_dist="uniform", shot_lo=10, shot_hi=40,
+                           name=cfg.name + "[sentence units]")
+    if kind == "chunks":
+        c = chunk_tokens
+        S = (cfg.N - cfg.question_len) // c
+        return cfg.replace(S=S, shot_dist="uniform", shot_lo=c, shot_hi=c, question_len=cfg.N - c * S,
+                           name=cfg.name + f"[{c}-token chunks]")
+    return cfg
+
+
+def workload_config(cfg, world: int) -> dict:
+    """The `config` entry of the JSON line: the same for the GPU arm and the reference arm."""
+    k_gb = cfg.B * cfg.L * cfg.Hkv * cfg.N * cfg.d * 2 / 1e9
+    return {"workload": cfg.name, "B": cfg.B, "L": cfg.L, "H": cfg.H, "Hkv": cfg.Hkv, "d": cfg.d, "N": cfg.N,
+            "W": cfg.W, "S": cfg.S, "r_p": cfg.r_p,
+            "l2": "inputs (K alone %.1f GB) larger than the 126 MB L2; no flush" % k_gb,
+            "parallelism": f"{world} independent replica(s), one batch of prompts each"}
+
+
 def algorithmic_bytes(cfg, kept_count: np.ndarray) -> dict:
     """Bytes the method itself must move per step: all of K read once, and the kept K and V rows
     read and written once each (actual kept counts)."""
@@ -181,14 +204,7 @@ def run_ours(args):
     if args.batch or args.layers:       # reduced copies of the workload, for profiler captures only
         cfg = cfg.replace(B=args.batch or cfg.B, L=args.layers or cfg.L,
                           name=f"{cfg.name}[B={args.batch or cfg.B},L={args.layers or cfg.L}]")
-    if args.units == "sentences":       # same tensors' shapes, units of 10-40 tokens
-        cfg = cfg.replace(S=(cfg.N - cfg.question_len) // 25, shot_dist="uniform", shot_lo=10, shot_hi=40,
-                          name=cfg.name + "[sentence units]")
-    elif args.units == "chunks":        # fixed chunks of --chunk-tokens tokens (16); the remainder joins the question
-        c = args.chunk_tokens
-        S = (cfg.N - cfg.question_len) // c
-        cfg = cfg.replace(S=S, shot_dist="uniform", shot_lo=c, shot_hi=c, question_len=cfg.N - c * S,
-                          name=cfg.name + f"[{c}-token chunks]")
+    cfg = units_variant(cfg, args.units, args.chunk_tokens)
     dims = skv.make_dims(cfg.B, cfg.L, cfg.H, cfg.Hkv, cfg.d, cfg.N, cfg.W, cfg.S)
     pol = skv.make_policy(r_p=cfg.r_p)
     Q, K, V, off = wl.prefill_batch(cfg, dev)
@@ -277,9 +293,7 @@ def run_ours(args):
         "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16 in, f32 accumulate", "data": "synthetic",
-        "config": {"workload": cfg.name, "B": cfg.B, "L": cfg.L, "H": cfg.H, "Hkv": cfg.Hkv, "d": cfg.d, "N": cfg.N,
-                   "W": cfg.W, "S": cfg.S, "r_p": cfg.r_p, "l2": "inputs (K alone %.1f GB) larger than the 126 MB L2; no flush" % (ab["k_read"] / 1e9),
-                   "parallelism": f"{world} independent replica(s), one batch of prompts each"},
+        "config": workload_config(cfg, world),
         "roofline": roofline, "path": path, "clocks": clocks, "gpu_launches": int(launches),
     }
     if sustained:
@@ -307,6 +321,38 @@ def run_ours(args):
             "note": "same step with SHOTKV_FLAG_TOKEN_IMPORTANCE: per-token importance materialised (two passes over K)",
             "frac_of_measured_hbm_for_two_k_reads": round((ab["total"] + ab["k_read"]) / (tok_ms * 1e-3) / 1e9 / peak, 4)}
         del imp
+    # ---------------- the same tensors with sentence-sized units and with fixed 16-token chunks as the
+    # semantic units (only the boundaries change): the paper's document-QA adaptation and chunk-level
+    # retention.  Short timed regions; the routes they take are chosen by the library.
+    if not args.no_units and args.units == "shots":
+        result["short_units"] = {}
+        for kind in ("sentences", "chunks"):
+            cu = units_variant(cfg, kind, args.chunk_tokens)
+            off_u = wl.all_shot_offsets(cu)
+            dims_u = skv.make_dims(cu.B, cu.L, cu.H, cu.Hkv, cu.d, cu.N, cu.W, cu.S)
+            M_u = skv.shotkv_kept_capacity(dims_u, pol, off_u)
+            out_u = skv.alloc_prefill_outputs(dims_u, M_u, device=dev)
+
+            def unit_step():
+                skv.shotkv_prefill_compress(ctx, dims_u, pol, Q, K, V, off_u, out_u["shot_scores"], out_u["keep"], out_u["kept_idx"],
+                                            out_u["kept_count"], M_u, out_u["Kc"], out_u["Vc"], None, 0, out_u["ws"])
+            for _ in range(3):
+                unit_step()
+            barrier(world)
+            n_u = max(3, min(args.steps, 20))
+            u0, u1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            u0.record()
+            for _ in range(n_u):
+                unit_step()
+            u1.record()
+            barrier(world)
+            u_ms = max_over_ranks(u0.elapsed_time(u1), world, dev) / n_u
+            ab_u = algorithmic_bytes(cu, out_u["kept_count"].cpu().numpy())
+            result["short_units"][kind] = {"units_per_prompt": cu.S, "ms_per_step": round(u_ms, 4), "steps": n_u,
+                                           "value": round(tokens / (u_ms * 1e-3), 1), "unit": UNIT,
+                                           "path_frac_of_measured_hbm": round(ab_u["total"] / (u_ms * 1e-3) / 1e9 / peak, 4)}
+            del out_u
+        torch.cuda.empty_cache()
     # ---------------- end to end from host buffers (rank-local, same workload)
     if not args.no_e2e:
         result["e2e"] = e2e_leg(skv, ctx, cfg, dims, pol, Q, K, V, off, Mcap, world, dev, args)
@@ -599,8 +645,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": args.gpus,
             "steps": steps, "warmup": warm, "ms_per_step": round(sec * 1e3, 2), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg.name, "B": cfg.B, "L": cfg.L, "H": cfg.H, "Hkv": cfg.Hkv, "d": cfg.d, "N": cfg.N,
-                       "W": cfg.W, "S": cfg.S, "r_p": cfg.r_p},
+            "config": workload_config(cfg, args.gpus),
             "cpu_baseline": {"value": round(value, 2), "unit": UNIT, "kind": "oracle", "cores": oracle_threads(),
                              "sample": f"each step = one (prompt, layer) unit of {cfg.name} ({cfg.N} token-layers); "
                                        f"tokens/s scaled by L = {cfg.L} layers per prompt"},
@@ -633,6 +678,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-units", action="store_true", help="skip the sentence-unit and chunk-unit forms of the step")
     ap.add_argument("--no-sustained", action="store_true", help="skip the seconds-long repeat of the step")
     args = ap.parse_args()
     if args.impl == "reference":
