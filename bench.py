@@ -45,7 +45,7 @@ FALLBACK_HBM_GBS = 6650.0
 # byte of the scoring kernel and of the two decode score kernels, taken on reduced copies of the
 # workloads (config 3 with B=1, L=8; config 4 with B=2) and scaled by the bytes of a full launch.
 # A ratio is set to None whenever its kernel has changed since its capture.
-SCORE_TC_TRAFFIC_RATIO = 1.043
+SCORE_TC_TRAFFIC_RATIO = 1.042
 DECODE_TRAFFIC_RATIO = 1.012
 DECODE_ATTEND_TRAFFIC_RATIO = 1.006
 NOMINAL_HBM_GBS = 8000.0
