@@ -36,7 +36,10 @@ struct ScoreFastCfg {
     static constexpr int kSubBytes = 128 * 128;
     static constexpr int kQBytes = kSub * kSubBytes;
     static constexpr int kStageBytes = kSub * kSubBytes;
-    static constexpr int kStages = D == 128 ? 5 : 6;
+    // An even number: the two MMA threads take alternate tiles, so with an even ring each of them meets
+    // a given stage every time round and its parity wait can never be a whole turn behind the barrier.
+    // (Four 32 KB stages measure the same as five.)
+    static constexpr int kStages = D == 128 ? 4 : 6;
     static constexpr int kBarBytes = 2048;
     static constexpr int kRingDepth = 4;                       // hand-over slots between a row's column slices
     static constexpr int kRings = 4;                           // one per warp quarter

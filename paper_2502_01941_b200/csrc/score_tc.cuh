@@ -453,6 +453,9 @@ __device__ __forceinline__ void mma_role(const Pipe<Cfg>& pp, const ScoreTcParam
                                          int which) {
     constexpr int NSUB = Cfg::kSub, KSTEPS = D / 16, NST = Cfg::kStages, TN = kTileKeys;
     constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TN >> 3) << 17) | ((128u >> 4) << 24);
+    // a thread that met a stage only every other turn of the ring would wait on a parity the barrier may
+    // already have passed twice
+    static_assert(NT == 1 || NST % NT == 0, "each MMA thread must meet every stage it uses on every turn of the K ring");
     int stage = 0, acc = 0, cur_u = -1;
     uint32_t fphase = 0, qfphase = 0, tephase0 = 1, tephase1 = 1;
     bool ok = true;
