@@ -41,6 +41,8 @@ from paper_2502_01941_b200 import workloads as wl
 METRIC = "prompt tokens compressed/sec"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0            # an earlier burst measurement on this machine, used only without MEASURED_PEAKS.json
+FALLBACK_BF16_TFLOPS_SUSTAINED = 1400.0  # the same, back to back under the power cap
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, one ncu capture each) per algorithmic
 # byte of the scoring kernel and of the two decode score kernels, taken on reduced copies of the
 # workloads (config 3 with B=1, L=8; config 4 with B=2) and scaled by the bytes of a full launch.
@@ -62,6 +64,17 @@ def measured_peaks():
         return float(p["hbm_gbs"]), "measured"
     except Exception:
         return FALLBACK_HBM_GBS, "fallback"
+
+
+def measured_tensor_peaks():
+    """Dense bf16 matmul throughput of this machine's B200s in TFLOP/s: (burst, sustained, source)."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["bf16_tflops"]), float(p["bf16_tflops_sustained"]), "measured"
+    except Exception:
+        return FALLBACK_BF16_TFLOPS, FALLBACK_BF16_TFLOPS_SUSTAINED, "fallback"
 
 
 class ClockSampler:
@@ -267,19 +280,38 @@ def run_ours(args):
     fast_name = "score_stream_kernel" if cfg.G * cfg.W > 128 else "score_fast_kernel"
     kernel_name = {"fast": fast_name, "exact": "score_tc_kernel"}[args.scoring] + \
         " (window QK^T on tcgen05 + softmax partials), one launch per step"
-    roofline = {"bound": "hbm", "kernel": kernel_name,
-                "achieved": round(achieved, 1), "peak": peak, "peak_source": peak_src, "unit": "GB/s",
-                "frac": round(achieved / peak, 4),
-                # measured DRAM bytes per launch: the captured ratio times the K bytes of a full launch
-                "traffic": int(SCORE_TC_TRAFFIC_RATIO * ab["k_read"]) if SCORE_TC_TRAFFIC_RATIO and args.scoring == "fast" else None,
-                "algorithmic_bytes_per_launch": ab["k_read"], "ms_per_launch": round(score_ms, 4),
-                # what actually limits this kernel: one exponential per logit.  16 per clock per SM is what
-                # the special-function unit alone delivers (measured); the kernel takes 5 of every 16
-                # column pairs on the FMA pipe instead, so the fraction may pass 1
-                "also": {"bound": "alu", "unit": "exp/clk/SM", "achieved": round(ex2_rate, 2), "peak": 16.0,
-                         "frac": round(ex2_rate / 16.0, 4), "at_sm_mhz": sm_mhz,
-                         "cycles_per_tile": round(rate_ms * 1e-3 * sm_mhz * 1e6 / tiles_per_sm, 1),
-                         "region": "sustained" if sustained else "steps"}}
+    # The scoring kernel is a contraction (Q K^T: 2 d flops per window logit) fed by one pass over K,
+    # followed by one exponential per logit.  Its roofline is the slower of the two machine limits:
+    # K bytes / copy bandwidth, or flops / the bf16 matmul rate this GPU sustains under its power cap
+    # (the steps run back to back at the cap, so the sustained figure is the one that applies; the
+    # fraction of the burst figure is given beside it).
+    flops = 2.0 * logits * cfg.d
+    tf_burst, tf_sustained, tf_src = measured_tensor_peaks()
+    achieved_tf = flops / (score_ms * 1e-3) / 1e12
+    hbm_rec = {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "peak_source": peak_src, "unit": "GB/s",
+               "frac": round(achieved / peak, 4), "floor_ms": round(ab["k_read"] / peak / 1e6, 4)}
+    tensor_rec = {"bound": "tensor", "achieved": round(achieved_tf, 1), "peak": tf_sustained,
+                  "peak_source": tf_src + ", sustained bf16 matmul", "unit": "TFLOP/s",
+                  "frac": round(achieved_tf / tf_sustained, 4), "frac_of_burst_peak": round(achieved_tf / tf_burst, 4),
+                  "floor_ms": round(flops / tf_sustained / 1e9, 4)}
+    # one exponential per logit: 16 per clock per SM is what the special-function unit alone delivers
+    # (measured); the kernel takes 5 of every 16 column pairs on the FMA pipe instead, so this
+    # fraction may pass 1
+    alu_rec = {"bound": "alu", "unit": "exp/clk/SM", "achieved": round(ex2_rate, 2), "peak": 16.0,
+               "frac": round(ex2_rate / 16.0, 4), "at_sm_mhz": sm_mhz,
+               "cycles_per_tile": round(rate_ms * 1e-3 * sm_mhz * 1e6 / tiles_per_sm, 1),
+               "region": "sustained" if sustained else "steps"}
+    first, second = (tensor_rec, hbm_rec) if tensor_rec["floor_ms"] > hbm_rec["floor_ms"] else (hbm_rec, tensor_rec)
+    roofline = dict(first)
+    roofline.update({
+        "kernel": kernel_name,
+        # measured DRAM bytes per launch: the captured ratio times the K bytes of a full launch (the capture
+        # was of the streaming kernel on config 3's shape with shots as units; null for anything else)
+        "traffic": int(SCORE_TC_TRAFFIC_RATIO * ab["k_read"]) if SCORE_TC_TRAFFIC_RATIO and args.scoring == "fast"
+        and args.workload == 3 and args.units == "shots" else None,
+        "algorithmic_bytes_per_launch": ab["k_read"], "algorithmic_flops_per_launch": int(flops),
+        "ms_per_launch": round(score_ms, 4),
+        "also": [second, alu_rec]})
     path = {"bytes_per_step": ab["total"], "k_read_bytes": ab["k_read"], "kv_gathered_bytes": ab["kv_gathered"],
             "achieved_gbs": round(ab["total"] / (ms_step * 1e-3) / 1e9, 1),
             "frac_of_measured_hbm": round(ab["total"] / (ms_step * 1e-3) / 1e9 / peak, 4),
