@@ -31,7 +31,7 @@ struct ColsumTcCfg {
     static constexpr int kSubBytes = 128 * 128;
     static constexpr int kQBytes = MB * kSub * kSubBytes;
     static constexpr int kStageBytes = kSub * kSubBytes;
-    static constexpr int kStages = D == 128 ? (MB == 2 ? 4 : 5) : 6;
+    static constexpr int kStages = D == 128 ? 4 : 6;              // even: see mma_role_transposed
     static constexpr int kBarBytes = 1024;
     static constexpr int kRows = 128 * MB;
     // per epilogue warp: the constants of its half of the rows, [rows/4] float4 (-M_r, -M_r+1, 1/Z_r, 1/Z_r+1)
@@ -51,6 +51,8 @@ __device__ __forceinline__ void mma_role_transposed(const Pipe<Cfg>& pp, const S
                                                     int item_end, int which) {
     constexpr int KSTEPS = D / 16, NST = Cfg::kStages, TN = kTileKeys, NR = 128 * MB;
     constexpr uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NR >> 3) << 17) | ((128u >> 4) << 24);
+    // two threads on alternate tiles: only an even ring lets each meet every stage it uses on every turn
+    static_assert(NST % 2 == 0, "each MMA thread must meet every stage it uses on every turn of the K ring");
     int stage = 0, acc = 0, cur_u = -1;
     uint32_t fphase = 0, qfphase = 0, tephase0 = 1, tephase1 = 1;
     bool ok = true;
