@@ -48,6 +48,7 @@ FALLBACK_BF16_TFLOPS_SUSTAINED = 1400.0  # the same, back to back under the powe
 # workloads (config 3 with B=1, L=8; config 4 with B=2) and scaled by the bytes of a full launch.
 # A ratio is set to None whenever its kernel has changed since its capture.
 SCORE_TC_TRAFFIC_RATIO = 1.042
+SCORE_FAST_TRAFFIC_RATIO = 1.021      # the 128-row kernel on config 2 at full size
 DECODE_TRAFFIC_RATIO = 1.012
 DECODE_ATTEND_TRAFFIC_RATIO = 1.006
 NOMINAL_HBM_GBS = 8000.0
@@ -286,6 +287,7 @@ def run_ours(args):
     # (the steps run back to back at the cap, so the sustained figure is the one that applies; the
     # fraction of the burst figure is given beside it).
     flops = 2.0 * logits * cfg.d
+    traffic_ratio = {3: SCORE_TC_TRAFFIC_RATIO, 2: SCORE_FAST_TRAFFIC_RATIO}.get(args.workload)
     tf_burst, tf_sustained, tf_src = measured_tensor_peaks()
     achieved_tf = flops / (score_ms * 1e-3) / 1e12
     hbm_rec = {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "peak_source": peak_src, "unit": "GB/s",
@@ -305,10 +307,9 @@ def run_ours(args):
     roofline = dict(first)
     roofline.update({
         "kernel": kernel_name,
-        # measured DRAM bytes per launch: the captured ratio times the K bytes of a full launch (the capture
-        # was of the streaming kernel on config 3's shape with shots as units; null for anything else)
-        "traffic": int(SCORE_TC_TRAFFIC_RATIO * ab["k_read"]) if SCORE_TC_TRAFFIC_RATIO and args.scoring == "fast"
-        and args.workload == 3 and args.units == "shots" else None,
+        # measured DRAM bytes per launch: the captured ratio times the K bytes of a full launch (captures
+        # exist for config 3's shape and for config 2, with shots as units; null for anything else)
+        "traffic": int(traffic_ratio * ab["k_read"]) if traffic_ratio and args.scoring == "fast" and args.units == "shots" else None,
         "algorithmic_bytes_per_launch": ab["k_read"], "algorithmic_flops_per_launch": int(flops),
         "ms_per_launch": round(score_ms, 4),
         "also": [second, alu_rec]})
