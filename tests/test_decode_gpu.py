@@ -271,3 +271,28 @@ def test_random_decode_shapes(ctx, cfg, M, protect, attend):
         counts, M = np.zeros((cfg.B, cfg.L), np.int32), 4
     units = [(b, l) for b in range(cfg.B) for l in range(cfg.L)]
     assert lockstep(ctx, cfg, M, units, counts, attend=attend, protect_recent=protect) <= 3
+
+
+@pytest.mark.parametrize("attend", [False, True], ids=["plain", "attend"])
+def test_decode_config4_runs_repeat_bit_exactly(ctx, attend):
+    """Every reduction on the decode path has a fixed order, so two runs over the same bytes must
+    agree bit for bit: config 4's shape for four eviction cycles, run twice from the same start;
+    accumulated scores, survivors, the decode region and (fused step) the attention outputs of
+    every sequence and layer are compared after each step."""
+    cfg = wl.DECODE_CONFIG
+    Kc, kept = wl.random_prefill_cache(cfg, 3276, "cuda")
+    Vc = wl.random_prefill_values(cfg, 3276, "cuda") if attend else None
+    a = GpuDecoder(ctx, cfg, Kc, kept, Vc=Vc)
+    b = GpuDecoder(ctx, cfg, Kc, kept, Vc=Vc)
+    for s in range(4 * cfg.recompress_every + 3):
+        q, k, v = wl.decode_step_inputs(cfg, s, "cuda")
+        a.step(q, k, v)
+        b.step(q, k, v)
+        torch.cuda.synchronize()
+        assert a.state.n_dec == b.state.n_dec and a.state.T == b.state.T
+        assert torch.equal(a.acc, b.acc), f"step {s}: accumulated scores differ between two runs"
+        assert torch.equal(a.born, b.born), f"step {s}: survivors differ between two runs"
+        if attend:
+            assert torch.equal(a.out, b.out), f"step {s}: attention outputs differ between two runs"
+    n = a.state.n_dec
+    assert torch.equal(a.Kd[:, :, :, :n], b.Kd[:, :, :, :n]) and torch.equal(a.Vd[:, :, :, :n], b.Vd[:, :, :, :n])
